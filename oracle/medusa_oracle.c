@@ -659,6 +659,46 @@ static int argmax_f(const float *v, int n)
  * sample argmax_v fl32(fl32(logits[last][v] * inv_tau) + gumbel[v]) with inv_tau = fl32(1/tau).
  * min_margin (nullable): smallest |P - thr| / thr over all typical decisions taken (conditioning report).
  */
+/*
+ * One typical-acceptance decision (Sec. 2.3.1): with l = row/tau, P = softmax(l) and Hn its entropy in nats,
+ * the candidate token passes iff P[token] > min(eps, delta * exp(-Hn)) (strict).  The three quantities of the
+ * criterion are returned so that hand-worked vectors can pin each of them, not only the decision.
+ */
+static int typical_decision(const float *lp, int V, double tau, double eps, double delta, int token, double *p_out,
+                            double *ent_out, double *thr_out)
+{
+    double mx = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        double l = (double)lp[v] / tau;
+        if (l > mx)
+            mx = l;
+    }
+    double se = 0.0;
+    for (int v = 0; v < V; ++v)
+        se += exp((double)lp[v] / tau - mx);
+    double lse = mx + log(se);
+    double ent = 0.0; /* H = -sum p log p */
+    for (int v = 0; v < V; ++v) {
+        double l = (double)lp[v] / tau;
+        double pv = exp(l - lse);
+        if (pv > 0.0)
+            ent -= pv * (l - lse);
+    }
+    double pc = exp((double)lp[token] / tau - lse);
+    double thr = fmin(eps, delta * exp(-ent));
+    *p_out = pc;
+    *ent_out = ent;
+    *thr_out = thr;
+    return pc > thr;
+}
+
+/* The same decision for one logits row, exported for the pins: returns 1 if `token` passes. */
+int32_t ora_typical_decision(const float *row, int32_t V, double tau, double eps, double delta, int32_t token,
+                             double *p_out, double *entropy_out, double *threshold_out)
+{
+    return typical_decision(row, V, tau, eps, delta, token, p_out, entropy_out, threshold_out);
+}
+
 void ora_evaluate_posterior(const float *logits, int32_t V, const int32_t *tree_tok, const int32_t *retrieve, int32_t P,
                             int32_t depth, int32_t mode, double tau, double eps, double delta, const float *gumbel,
                             int32_t *best, int32_t *accept_len, int32_t *next_root, int32_t *acc_nodes,
@@ -681,26 +721,8 @@ void ora_evaluate_posterior(const float *logits, int32_t V, const int32_t *tree_
             if (mode == 0) {
                 ok = tree_tok[c] == argmax_f(lp, V);
             } else {
-                double mx = -INFINITY;
-                for (int v = 0; v < V; ++v) {
-                    double l = (double)lp[v] / tau;
-                    if (l > mx)
-                        mx = l;
-                }
-                double se = 0.0;
-                for (int v = 0; v < V; ++v)
-                    se += exp((double)lp[v] / tau - mx);
-                double lse = mx + log(se);
-                double ent = 0.0; /* H = -sum p log p = lse - sum p l */
-                for (int v = 0; v < V; ++v) {
-                    double l = (double)lp[v] / tau;
-                    double pv = exp(l - lse);
-                    if (pv > 0.0)
-                        ent -= pv * (l - lse);
-                }
-                double pc = exp((double)lp[tree_tok[c]] / tau - lse);
-                double thr = fmin(eps, delta * exp(-ent));
-                ok = pc > thr;
+                double pc, ent, thr;
+                ok = typical_decision(lp, V, tau, eps, delta, tree_tok[c], &pc, &ent, &thr);
                 if (thr > 0.0) {
                     double mg = fabs(pc - thr) / thr;
                     if (mg < mm)

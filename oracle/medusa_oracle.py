@@ -299,6 +299,17 @@ def evaluate_posterior(logits_f32, tree_tok, tree, mode=GREEDY, tau=0.0, eps=0.0
                 min_margin=margin.value)
 
 
+def typical_decision(row_f32, token, tau, eps, delta):
+    """One typical-acceptance decision on one logits row -> dict(ok, p, H, threshold) (the oracle's own numbers)."""
+    row = _f32(row_f32)
+    pc, ent, thr = C.c_double(), C.c_double(), C.c_double()
+    fn = lib().ora_typical_decision
+    fn.restype = C.c_int32
+    ok = fn(_p(row), C.c_int32(row.size), C.c_double(tau), C.c_double(eps), C.c_double(delta), C.c_int32(int(token)),
+            C.byref(pc), C.byref(ent), C.byref(thr))
+    return dict(ok=bool(ok), p=pc.value, H=ent.value, threshold=thr.value)
+
+
 def accept_and_update_kv(tree_k, tree_v, k_cache, v_cache, acc_nodes, accept_len, max_commit, L, hidden, tree_tok):
     """In-place on the float64 caches.  -> dict(L, h_last, emitted, moved_src, moved_dst)"""
     NL, T, H, D = tree_k.shape

@@ -459,6 +459,20 @@ def test_typical_acceptance_hand_vectors(oracle):
                                           delta=c["delta"])
             assert (r["accept_len"] == 1) == c["pass"][x], (c, x)
             assert r["acc_nodes"].tolist() == ([0, 1] if c["pass"][x] else [0, -1])
+            # the three quantities of the criterion, as the oracle itself evaluates them, against the hand values
+            st = oracle.typical_decision(lg, x, c["tau"], c["eps"], c["delta"])
+            assert st["ok"] == c["pass"][x]
+            assert abs(st["p"] - c["p"][x]) < 2e-6, (c, x, st)
+            assert abs(st["H"] - c["H"]) < 2e-6, (c, st)
+            assert abs(st["threshold"] - c["threshold"]) < 2e-6, (c, st)
+            if "delta_exp_negH" in c:
+                assert abs(c["delta"] * math.exp(-st["H"]) - c["delta_exp_negH"]) < 2e-6
+        if c.get("entropy_branch_decides"):
+            # the entropy term is what decides: some token sits between delta*exp(-H) and eps, clear of both
+            # (>= 10 % above the threshold, >= 4 % below eps; >= 10 % on both sides in the tau = 1 cases)
+            thr = c["threshold"]
+            assert thr < c["eps"] / 1.1
+            assert any(1.1 * thr <= q <= c["eps"] / (1.1 if c["tau"] == 1.0 else 1.04) for q in c["p"])
 
 
 def _planted(oracle, t, path_row, n_ok, V=64, seed=0):
