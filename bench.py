@@ -51,11 +51,6 @@ WORKLOADS = {
                        "acceptance, batch 1)"),
 }
 WORKLOAD = WORKLOADS["7b"]
-# ncu DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel: the
-# launch-weighted mean over a step's 129 GEMM launches, from the capture summarised in
-# profiles/gemm_tc_kernel_7b_2layers.md (the four layer shapes captured on a 2-layer model of the same width;
-# a layer's traffic does not depend on the depth, the LM head's 266 MB is its weights plus logits).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 108.3e6
 
 
 def measured_peaks():
@@ -198,6 +193,9 @@ def run_reference(args):
         "metric": WORKLOAD["metric"], "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+        # each timed step runs 1 of the identical decoder layers; ms_per_step is that sample scaled to the full depth,
+        # so steps x ms_per_step exceeds the wall time of this run by design
+        "extrapolated": True, "layers_run_per_step": 1, "layers_total": cfg["n_layers"],
         "config": {"workload": WORKLOAD["name"], "tree_nodes": 64, "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"]},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -207,6 +205,26 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------------------------- GPU arm
+
+def measure_read_peak(torch, B, stream, gib: float = 4.0, reps: int = 5):
+    """Read-only DRAM bandwidth of this GPU, GB/s: one pass of 16-byte streaming loads over a buffer far larger than
+    the L2, best of `reps`, CUDA events on the stream the kernel runs on."""
+    n = int(gib * (1 << 30))
+    buf = torch.empty(n, dtype=torch.uint8, device="cuda")
+    buf.random_(0, 255)
+    sink = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    best = 0.0
+    for i in range(reps + 2):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        B.stream_read(buf, n, sink, stream.cuda_stream)
+        b.record(stream)
+        b.synchronize()
+        if i >= 2:
+            best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
+    del buf
+    return best
+
 
 def run_gpu(args):
     import torch
@@ -289,6 +307,7 @@ def run_gpu(args):
         step_e2e()
     for _ in range(args.warmup):
         step_device_only()
+    read_peak_gbs = measure_read_peak(torch, B, stream)
     L0 = ctx.state()["cache_len"]
     ctx.get_profile(reset=True)
     sampler = ClockSampler(local)
@@ -367,6 +386,7 @@ def run_gpu(args):
             kernels["heads_gemv"]["achieved_gbs"] = R.heads_bytes(cfg["d"], cfg["vocab"], tree["depth"]) / (
                 kernels["heads_gemv"]["ms_per_step"] * 1e-3) / 1e9
         kernels["gemm"]["achieved_gbs"] = achieved
+        traffic, traffic_note = R.captured_traffic("gemm_tc_kernel", WORKLOAD["model"])
         line = {
             "metric": WORKLOAD["metric"],
             "value": tokens / (ms * 1e-3),
@@ -398,11 +418,15 @@ def run_gpu(args):
             "step_graphs": dict(ctx.step_graph_info(), note="kernel launches replayed from whole-step CUDA graphs the "
                                                             "library captured; gpu_launches counts the kernels inside them"),
             "step_roofline": {"bytes_per_step": sb["total"], "achieved_gbs": step_gbs, "frac_of_measured": step_gbs / peaks["hbm_gbs"],
+                              "frac_of_read_peak": step_gbs / read_peak_gbs if read_peak_gbs else None,
                               "frac_of_8tbs_nominal": step_gbs / 8000.0, "peak_source": peaks["source"]},
+            "read_peak": {"gbs": read_peak_gbs, "how": "16-byte streaming loads over 4 GiB, nothing written, best of 5, CUDA "
+                                                       "events; measured in this run before the timed regions"},
             "roofline": {"kernel": "backbone GEMM (M = 64 tree tokens), %d launches per step" % round(gemm_launches_step),
                          "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"],
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if WORKLOAD["model"] == "7b" else None,
+                         "frac_of_read_peak": achieved / read_peak_gbs if read_peak_gbs else None,
+                         "traffic": traffic, "traffic_note": traffic_note,
                          "bytes_per_step": gemm_bytes_step, "ms_per_step": gemm_ms_step, "peak_source": peaks["source"],
                          "timing": "CUDA events around every launch in an instrumented repeat of the timed steps"},
             "kernels": kernels,
@@ -420,6 +444,19 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def spawn_replicas(n: int) -> int:
+    """`bench.py --gpus N` started without a launcher: start the N single-GPU replicas ourselves (one process per GPU,
+    rendezvous on 127.0.0.1) and pass their exit code on."""
+    import socket
+
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -431,6 +468,13 @@ def main():
     global WORKLOAD
     WORKLOAD = WORKLOADS[args.workload]
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus))
+    if world != args.gpus:
+        raise SystemExit("--gpus %d does not match the launcher's WORLD_SIZE=%d" % (args.gpus, world))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -100,7 +100,30 @@ enum {
     MEDUSA_WS_ACC_NODES = 9, /* int32 [depth+1] */
     MEDUSA_WS_STATE = 10,   /* int32 [8]: cache_len, root, best, accept_len, next_root, n_emitted, status, steps */
     MEDUSA_WS_H_LAST = 11,  /* float [d] */
-    MEDUSA_WS_EMITTED = 12  /* int32 [depth+1] */
+    MEDUSA_WS_EMITTED = 12, /* int32 [depth+1] */
+    /* copies taken at the layer chosen with MEDUSA_OPT_LAYER_TAP during the last backbone pass (64 rows, T used): */
+    MEDUSA_WS_TAP_X_IN = 13,   /* float [64][d]  residual stream entering the layer */
+    MEDUSA_WS_TAP_X_OUT = 14,  /* float [64][d]  residual stream leaving it */
+    MEDUSA_WS_TAP_ATT = 15,    /* dtype [P][64][H*D] the layer's attention output as the output projection reads it
+                                * (bf16 model: P = 2 planes whose sum is the value; f32 model: P = 1) */
+    MEDUSA_WS_TAP_XN_OUT = 16  /* dtype [P][64][d] RMSNorm of X_OUT with the gain of the norm that follows the layer
+                                * (the next layer's attention norm, or the final norm after the last layer) */
+};
+
+/* Context options for medusa_set_option. */
+enum {
+    MEDUSA_OPT_STEP_GRAPHS = 0,      /* 1 (default): medusa_decode_step may capture and replay whole-step CUDA graphs; 0: never */
+    MEDUSA_OPT_ATTENTION_KERNEL = 1, /* bf16 / head_dim 128 tree attention: 0 automatic (default), 1 mma.sync, 2 tcgen05 */
+    MEDUSA_OPT_ATTENTION_LENGTH_HINT = 2, /* host-side upper bound of *cache_len for medusa_tree_attention (kernel choice and
+                                           * grid size follow it; a longer cache is still processed completely); < 0: L_max */
+    MEDUSA_OPT_LAYER_TAP = 3,        /* layer whose input / attention output / output the next passes copy to the TAP
+                                      * buffers (parity checks layer by layer); -1 (default) off */
+    MEDUSA_OPT_SPIN_LIMIT = 4,       /* polls after which a bounded device-side wait gives up with MEDUSA_ERR_TIMEOUT;
+                                      * 0 = the kernels' default (about 4 million) */
+    MEDUSA_OPT_WITHHOLD_LOAD = 5     /* failure-path test hook, one shot: 1 = in the next tensor-core GEMM launch, 2 = in the
+                                      * next tcgen05 attention launch, one CTA's producer issues no load at all, so that its
+                                      * consumers' bounded waits expire with nothing in flight; the launch returns, its output
+                                      * is unusable and the device status becomes MEDUSA_ERR_TIMEOUT */
 };
 
 /* ---- lifetime ------------------------------------------------------------------------------------ */
@@ -120,6 +143,10 @@ const void *medusa_workspace_ptr(medusa_ctx *ctx, int32_t which);
  * dst_host. */
 int32_t medusa_read_workspace(medusa_ctx *ctx, int32_t which, int64_t offset_bytes, void *dst_host, int64_t bytes);
 
+/* Sets one of the MEDUSA_OPT_* options.  Options that captured step graphs depend on synchronise the stream and drop
+ * those graphs.  Errors: INVALID_ARG (unknown option, value out of range). */
+int32_t medusa_set_option(medusa_ctx *ctx, int32_t option, int64_t value);
+
 /* Kernel-launch accounting and optional per-category device timing (CUDA events around every launch; adds
  * event overhead, so leave it off when timing whole steps).  Categories: 0 GEMM, 1 tree attention,
  * 2 Medusa-head GEMV, 3 element-wise (embed, RMSNorm, RoPE, SwiGLU), 4 top-k + candidate expansion,
@@ -131,6 +158,13 @@ int32_t medusa_set_profiling(medusa_ctx *ctx, int32_t on);
  * context was created (host int, nullable). */
 int32_t medusa_step_graph_info(const medusa_ctx *ctx, int32_t *n_graphs_host, int64_t *n_replays_host);
 int32_t medusa_get_profile(medusa_ctx *ctx, double *ms_host, int64_t *launches_host, int32_t reset);
+
+/* Measurement aid (the paper has no counterpart): enqueues on `stream` (a cudaStream_t on the calling thread's current
+ * device) a kernel that reads the first `bytes` bytes of device buffer `buf` (16-byte aligned) once with 16-byte
+ * streaming loads and writes at most `sink_floats` floats to device buffer `sink`.  Timed with CUDA events over a buffer
+ * much larger than the L2 it gives the read-only DRAM bandwidth, the ceiling for kernels that read far more than
+ * they write.  Errors: INVALID_ARG, CUDA. */
+int32_t medusa_stream_read(const void *buf, int64_t bytes, float *sink, int32_t sink_floats, void *stream);
 
 /* ---- a0: static tree (paper Sec. 2.1.2 Fig. 2; Sec. 2.3.3 for the sparse tree) -------------------- */
 
@@ -258,7 +292,9 @@ int32_t medusa_tree_pass(medusa_ctx *ctx, const int32_t *tokens);
  * same launch configuration (acceptance parameters, min(max_commit, depth + 1), presence of gumbel, the two host
  * pointers; the cache length is read on the device) is captured into a CUDA graph, and later steps with that
  * configuration replay it (up to 16 graphs per context; pageable host pointers, a stream that is itself being
- * captured, profiling and MEDUSA_STEP_GRAPH=0 keep the plain launches).  A replayed step reads its noise row
+ * captured, profiling and MEDUSA_OPT_STEP_GRAPHS = 0 keep the plain launches).
+ * When max_commit cuts the accepted path short, the next step's root is the path's next (already accepted) token,
+ * so repeated calls with a small max_commit continue the same token stream.  A replayed step reads its noise row
  * from a buffer of the context, into which gumbel is copied first. */
 int32_t medusa_decode_step(medusa_ctx *ctx, const medusa_accept_params *params, const float *gumbel,
                            int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host);

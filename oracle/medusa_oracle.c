@@ -577,6 +577,87 @@ static inline int kv_heads(const void *model)
  *   hidden        : [T][d]  final-norm output (the LM head's input, and the Medusa heads' input)
  *   logits        : [T][V]  (nullable)
  */
+/* A value as a bfloat16 store holds it: rounded to float, then to the nearest bfloat16 (ties to even). */
+static double round_bf16(double v)
+{
+    float f = (float)v;
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7f800000u) == 0x7f800000u)
+        return (double)f; /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Scratch of one layer evaluation. */
+typedef struct {
+    double *n, *q, *att, *o, *g, *u;
+} layer_scratch;
+
+static void layer_scratch_alloc(layer_scratch *s, int T, int d, int hd, int F)
+{
+    s->n = (double *)malloc((size_t)T * d * sizeof(double));
+    s->q = (double *)malloc((size_t)T * hd * sizeof(double));
+    s->att = (double *)malloc((size_t)T * hd * sizeof(double));
+    s->o = (double *)malloc((size_t)T * d * sizeof(double));
+    s->g = (double *)malloc((size_t)T * F * sizeof(double));
+    s->u = (double *)malloc((size_t)T * F * sizeof(double));
+}
+
+static void layer_scratch_free(layer_scratch *s)
+{
+    free(s->n); free(s->q); free(s->att); free(s->o); free(s->g); free(s->u);
+}
+
+/*
+ * One pre-norm Llama block on T tree tokens (App. G Table 5, "parallel decoding"), in place on x [T][d]:
+ *   x += Wo Attn(RMSNorm(x));  x += Wd (SiLU(Wg n) * (Wu n)), n = RMSNorm(x).
+ * kc, vc: this layer's cache [Hkv][L_max][D]; tk, tv: this layer's rotated tree keys and values [T][Hkv][D] (written).
+ * kv_bf16 != 0: the tree keys (after rotation) and values are held as a bfloat16 KV cache holds them -- the rounding
+ * belongs to the workload's definition of its cache storage, not to the method.  The attention output is left in
+ * s->att.
+ */
+static void layer_forward(const ora_model *m, int l, double *x, const uint64_t *mask, const int32_t *pos, int T, int L,
+                          int L_max, const double *kc, const double *vc, double *tk, double *tv, int kv_bf16,
+                          layer_scratch *s)
+{
+    int d = m->d, H = m->n_heads, Hkv = kv_heads(m), D = m->head_dim, F = m->ffn, dt = m->wdtype;
+    int hd = H * D, hkd = Hkv * D;
+    const void *const *w = m->layers + (size_t)l * 9;
+    double *n = s->n, *q = s->q, *att = s->att, *o = s->o, *g = s->g, *u = s->u;
+    for (int t = 0; t < T; ++t)
+        rmsnorm(x + (size_t)t * d, w[0], dt, d, m->rms_eps, n + (size_t)t * d);
+    linear(w[1], dt, hd, d, n, T, d, q, hd);
+    linear(w[2], dt, hkd, d, n, T, d, tk, hkd);
+    linear(w[3], dt, hkd, d, n, T, d, tv, hkd);
+    for (int t = 0; t < T; ++t) {
+        for (int h = 0; h < H; ++h)
+            rope(q + ((size_t)t * H + h) * D, D, (int64_t)L + pos[t], m->rope_theta);
+        for (int h = 0; h < Hkv; ++h)
+            rope(tk + ((size_t)t * Hkv + h) * D, D, (int64_t)L + pos[t], m->rope_theta);
+    }
+    if (kv_bf16)
+        for (size_t i = 0; i < (size_t)T * hkd; ++i) {
+            tk[i] = round_bf16(tk[i]);
+            tv[i] = round_bf16(tv[i]);
+        }
+    tree_attention_core(q, tk, tv, kc, vc, T, H, Hkv, D, L, L_max, mask, att, NULL);
+    linear(w[4], dt, d, hd, att, T, hd, o, d);
+    for (size_t i = 0; i < (size_t)T * d; ++i)
+        x[i] += o[i];
+    for (int t = 0; t < T; ++t)
+        rmsnorm(x + (size_t)t * d, w[5], dt, d, m->rms_eps, n + (size_t)t * d);
+    linear(w[6], dt, F, d, n, T, d, g, F);
+    linear(w[7], dt, F, d, n, T, d, u, F);
+    for (size_t i = 0; i < (size_t)T * F; ++i)
+        g[i] = silu(g[i]) * u[i];
+    linear(w[8], dt, d, F, g, T, F, o, d);
+    for (size_t i = 0; i < (size_t)T * d; ++i)
+        x[i] += o[i];
+}
+
 void ora_tree_pass(const ora_model *m, const int32_t *tokens, const uint64_t *mask, const int32_t *pos, int32_t T,
                    int32_t L, int32_t L_max, const double *kc, const double *vc, double *tree_k, double *tree_v,
                    double *hidden, double *logits)
@@ -584,55 +665,53 @@ void ora_tree_pass(const ora_model *m, const int32_t *tokens, const uint64_t *ma
     int d = m->d, H = m->n_heads, Hkv = kv_heads(m), D = m->head_dim, F = m->ffn, dt = m->wdtype;
     int hd = H * D, hkd = Hkv * D;
     double *x = (double *)malloc((size_t)T * d * sizeof(double));
-    double *n = (double *)malloc((size_t)T * d * sizeof(double));
-    double *q = (double *)malloc((size_t)T * hd * sizeof(double));
-    double *att = (double *)malloc((size_t)T * hd * sizeof(double));
-    double *o = (double *)malloc((size_t)T * d * sizeof(double));
-    double *g = (double *)malloc((size_t)T * F * sizeof(double));
-    double *u = (double *)malloc((size_t)T * F * sizeof(double));
+    layer_scratch s;
+    layer_scratch_alloc(&s, T, d, hd, F);
     for (int t = 0; t < T; ++t)
         for (int i = 0; i < d; ++i)
             x[(size_t)t * d + i] = wget(m->embed, (size_t)tokens[t] * d + i, dt);
-    for (int l = 0; l < m->n_layers; ++l) {
-        const void *const *w = m->layers + (size_t)l * 9;
-        double *tk = tree_k + (size_t)l * T * hkd, *tv = tree_v + (size_t)l * T * hkd;
-        for (int t = 0; t < T; ++t)
-            rmsnorm(x + (size_t)t * d, w[0], dt, d, m->rms_eps, n + (size_t)t * d);
-        linear(w[1], dt, hd, d, n, T, d, q, hd);
-        linear(w[2], dt, hkd, d, n, T, d, tk, hkd);
-        linear(w[3], dt, hkd, d, n, T, d, tv, hkd);
-        for (int t = 0; t < T; ++t) {
-            for (int h = 0; h < H; ++h)
-                rope(q + ((size_t)t * H + h) * D, D, (int64_t)L + pos[t], m->rope_theta);
-            for (int h = 0; h < Hkv; ++h)
-                rope(tk + ((size_t)t * Hkv + h) * D, D, (int64_t)L + pos[t], m->rope_theta);
-        }
-        tree_attention_core(q, tk, tv, kc + (size_t)l * Hkv * L_max * D, vc + (size_t)l * Hkv * L_max * D, T, H, Hkv, D,
-                            L, L_max, mask, att, NULL);
-        linear(w[4], dt, d, hd, att, T, hd, o, d);
-        for (size_t i = 0; i < (size_t)T * d; ++i)
-            x[i] += o[i];
-        for (int t = 0; t < T; ++t)
-            rmsnorm(x + (size_t)t * d, w[5], dt, d, m->rms_eps, n + (size_t)t * d);
-        linear(w[6], dt, F, d, n, T, d, g, F);
-        linear(w[7], dt, F, d, n, T, d, u, F);
-        for (size_t i = 0; i < (size_t)T * F; ++i)
-            g[i] = silu(g[i]) * u[i];
-        linear(w[8], dt, d, F, g, T, F, o, d);
-        for (size_t i = 0; i < (size_t)T * d; ++i)
-            x[i] += o[i];
-    }
+    for (int l = 0; l < m->n_layers; ++l)
+        layer_forward(m, l, x, mask, pos, T, L, L_max, kc + (size_t)l * Hkv * L_max * D, vc + (size_t)l * Hkv * L_max * D,
+                      tree_k + (size_t)l * T * hkd, tree_v + (size_t)l * T * hkd, 0, &s);
     for (int t = 0; t < T; ++t)
         rmsnorm(x + (size_t)t * d, m->final_norm, dt, d, m->rms_eps, hidden + (size_t)t * d);
     if (logits)
         linear(m->lm_head, dt, m->vocab, d, hidden, T, d, logits, m->vocab);
     free(x);
-    free(n);
-    free(q);
-    free(att);
-    free(o);
-    free(g);
-    free(u);
+    layer_scratch_free(&s);
+}
+
+/*
+ * Layer l alone on a given layer input (the same code the pass above runs): x [T][d] in/out, att_out [T][H*D]
+ * (nullable) receives the attention output, kc/vc are THIS layer's cache [Hkv][L_max][D], tk/tv [T][Hkv][D] are written.
+ * Used to check an implementation layer by layer on that implementation's own layer inputs and cache.
+ */
+void ora_layer(const ora_model *m, int32_t l, double *x, const uint64_t *mask, const int32_t *pos, int32_t T, int32_t L,
+               int32_t L_max, const double *kc, const double *vc, double *tk, double *tv, int32_t kv_bf16, double *att_out)
+{
+    layer_scratch s;
+    layer_scratch_alloc(&s, T, m->d, m->n_heads * m->head_dim, m->ffn);
+    layer_forward(m, l, x, mask, pos, T, L, L_max, kc, vc, tk, tv, kv_bf16, &s);
+    if (att_out)
+        memcpy(att_out, s.att, (size_t)T * m->n_heads * m->head_dim * sizeof(double));
+    layer_scratch_free(&s);
+}
+
+/* The closing steps of a pass on a given residual stream x [T][d]: hidden = final RMSNorm(x) (nullable out), then the
+ * LM head on `hidden_in` if that is given, else on the hidden just computed; logits [T][V] (nullable). */
+void ora_final_norm_lm_head(const ora_model *m, const double *x, const double *hidden_in, int32_t T, double *hidden,
+                            double *logits)
+{
+    int d = m->d;
+    double *hn = (double *)malloc((size_t)T * d * sizeof(double));
+    if (x)
+        for (int t = 0; t < T; ++t)
+            rmsnorm(x + (size_t)t * d, m->final_norm, m->wdtype, d, m->rms_eps, hn + (size_t)t * d);
+    if (hidden && x)
+        memcpy(hidden, hn, (size_t)T * d * sizeof(double));
+    if (logits)
+        linear(m->lm_head, m->wdtype, m->vocab, d, hidden_in ? hidden_in : hn, T, d, logits, m->vocab);
+    free(hn);
 }
 
 /* ------------------------------------------------------------------ acceptance */

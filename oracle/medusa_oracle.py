@@ -273,6 +273,39 @@ def tree_pass(model: Model, tokens, tree, L, k_cache, v_cache, want_logits=True)
     return dict(logits=logits, hidden=hidden, tree_k=tk, tree_v=tv)
 
 
+def layer(model: Model, l, x_in, tree, L, k_cache_l, v_cache_l, kv_bf16=False):
+    """Layer l alone on a given layer input x_in [T][d]; k_cache_l, v_cache_l: THIS layer's cache, float64
+    [Hkv][L_max][D].  kv_bf16: the tree keys/values are held as a bfloat16 cache holds them.
+    -> dict(x_out [T][d], att [T][H*D], tree_k, tree_v [T][Hkv][D]) float64"""
+    c = model.cfg
+    x = np.array(x_in, dtype=np.float64, order="C")
+    T = x.shape[0]
+    L_max = k_cache_l.shape[1]
+    assert k_cache_l.dtype == np.float64 and k_cache_l.flags.c_contiguous
+    assert v_cache_l.dtype == np.float64 and v_cache_l.flags.c_contiguous
+    tk = np.zeros((T, model.kv_heads, c["head_dim"]), dtype=np.float64)
+    tv = np.zeros_like(tk)
+    att = np.zeros((T, c["n_heads"] * c["head_dim"]), dtype=np.float64)
+    mask = np.ascontiguousarray(tree["mask"], dtype=np.uint64)
+    lib().ora_layer(C.byref(model.c), C.c_int32(int(l)), _p(x), _p(mask), _p(_i32(tree["pos"])), C.c_int32(T),
+                    C.c_int32(int(L)), C.c_int32(L_max), _p(k_cache_l), _p(v_cache_l), _p(tk), _p(tv),
+                    C.c_int32(1 if kv_bf16 else 0), _p(att))
+    return dict(x_out=x, att=att, tree_k=tk, tree_v=tv)
+
+
+def final_norm_lm_head(model: Model, x=None, hidden_in=None, want_logits=True):
+    """hidden = final RMSNorm(x) (if x is given); logits = LM head of hidden_in if given, else of that hidden."""
+    c = model.cfg
+    src = x if x is not None else hidden_in
+    T = np.asarray(src).shape[0]
+    xx = None if x is None else _f64(x)
+    hi = None if hidden_in is None else _f64(hidden_in)
+    hidden = np.zeros((T, c["d"]), dtype=np.float64) if x is not None else None
+    logits = np.zeros((T, c["vocab"]), dtype=np.float64) if want_logits else None
+    lib().ora_final_norm_lm_head(C.byref(model.c), _p(xx), _p(hi), C.c_int32(T), _p(hidden), _p(logits))
+    return dict(hidden=hidden, logits=logits)
+
+
 # ----------------------------------------------------------------------------- acceptance / commit
 
 GREEDY, TYPICAL = 0, 1

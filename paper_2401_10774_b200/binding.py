@@ -18,7 +18,9 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_CACHE_FULL, ERR_CUDA, ERR_T
 F32, BF16 = 0, 1
 GREEDY, TYPICAL = 0, 1
 (WS_LOGITS, WS_HIDDEN, WS_TREE_K, WS_TREE_V, WS_K_CACHE, WS_V_CACHE, WS_HEAD_LOGITS, WS_TOPK_IDX, WS_TREE_TOK,
- WS_ACC_NODES, WS_STATE, WS_H_LAST, WS_EMITTED) = range(13)
+ WS_ACC_NODES, WS_STATE, WS_H_LAST, WS_EMITTED, WS_TAP_X_IN, WS_TAP_X_OUT, WS_TAP_ATT, WS_TAP_XN_OUT) = range(17)
+(OPT_STEP_GRAPHS, OPT_ATTENTION_KERNEL, OPT_ATTENTION_LENGTH_HINT, OPT_LAYER_TAP, OPT_SPIN_LIMIT,
+ OPT_WITHHOLD_LOAD) = range(6)
 LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 
@@ -241,6 +243,9 @@ class Context:
         self._check(lib().medusa_get_profile(self.handle, _ptr(ms), _ptr(n), C.c_int32(1 if reset else 0)))
         return {k: dict(ms=float(ms[i]), launches=int(n[i])) for i, k in enumerate(self.PROF_NAMES)}
 
+    def set_option(self, option: int, value: int):
+        self._check(lib().medusa_set_option(self.handle, C.c_int32(option), C.c_int64(int(value))))
+
     def step_graph_info(self) -> dict:
         n, r = C.c_int32(0), C.c_int64(0)
         self._check(lib().medusa_step_graph_info(self.handle, C.byref(n), C.byref(r)))
@@ -264,6 +269,14 @@ class Context:
     def state(self) -> dict:
         s = self.read_workspace(WS_STATE, (8,), np.int32).tolist()
         return dict(cache_len=s[0], root=s[1], best=s[2], accept_len=s[3], next_root=s[4], n_emitted=s[5], status=s[6])
+
+
+def stream_read(buf, nbytes: int, sink, stream=None):
+    """medusa_stream_read: enqueue one read-only pass over `nbytes` bytes of device tensor `buf` (timing aid)."""
+    rc = lib().medusa_stream_read(_ptr(buf), C.c_int64(int(nbytes)), _ptr(sink), C.c_int32(int(sink.numel())),
+                                  C.c_void_p(0 if stream is None else int(stream)))
+    if rc != OK:
+        raise MedusaError(rc, "medusa_stream_read")
 
 
 def tree_attention_static(q, k_new, v_new, k_cache, v_cache, cache_len, mask, T, H, L_max, L_hint, out, lse=None,

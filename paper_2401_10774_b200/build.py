@@ -1,6 +1,9 @@
 """Builds the CUDA library in-tree with nvcc for sm_100a (cross-compiles without a GPU).
 
-    python -m paper_2401_10774_b200.build [--force] [--verbose]
+    python -m paper_2401_10774_b200.build [--force] [--verbose] [--timing-aids]
+
+--timing-aids compiles with -DMEDUSA_TIMING_AIDS: only such a build reads the MEDUSA_* environment switches used
+for comparison runs (ring depth, serialised launches, dropped kernel classes); the default build reads none.
 """
 from __future__ import annotations
 
@@ -34,9 +37,15 @@ def _newest_header() -> float:
     return t
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+def build_library(force: bool = False, verbose: bool = False, timing_aids: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
+    # a change of flavour rebuilds everything
+    stamp = os.path.join(OBJ, "flavour")
+    flavour = "timing-aids" if timing_aids else "default"
+    if not os.path.exists(stamp) or open(stamp).read() != flavour:
+        force = True
+    extra = ["-DMEDUSA_TIMING_AIDS"] if timing_aids else []
     hdr = _newest_header()
     jobs = []
     objs = []
@@ -45,7 +54,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         o = os.path.join(OBJ, os.path.splitext(src)[0] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-x", "cu", "-c", s, "-o", o]
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-x", "cu", "-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):
@@ -61,8 +70,10 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         tmp = LIB + ".%d.tmp" % os.getpid()
         run([nvcc, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
         os.replace(tmp, LIB)
+    with open(stamp, "w") as f:
+        f.write(flavour)
     return LIB
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv, timing_aids="--timing-aids" in sys.argv))

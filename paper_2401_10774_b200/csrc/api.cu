@@ -52,6 +52,15 @@ struct medusa_ctx {
     // ATTN_TC_MIN_L keys on, the mma.sync kernel otherwise), 1 = always mma.sync, 2 = always tcgen05
     // (MEDUSA_ATTENTION=mma_sync|tcgen05)
     int attn_mode = 0;
+    int attn_len_hint = -1;  // host-side bound of the cache length for the stand-alone attention call (< 0: the capacity)
+    // layer tap (MEDUSA_OPT_LAYER_TAP): copies of one layer's input, attention output and output, for parity checks
+    int tap_layer = -1;
+    float *tap_x_in = nullptr, *tap_x_out = nullptr;  // [64][d] residual stream before / after the layer
+    void *tap_att = nullptr;                          // the layer's attention output as the o projection reads it
+    void *tap_xn_out = nullptr;                       // normalised residual stream after the layer (next norm's gain)
+    // test hooks for the bounded device-side waits (MEDUSA_OPT_SPIN_LIMIT, MEDUSA_OPT_WITHHOLD_LOAD)
+    uint32_t spin_limit = 0;  // 0: the kernels' default
+    int withhold = 0;         // one-shot: 1 = next tensor-core GEMM launch, 2 = next tcgen05 attention launch
     // host-side upper bound of the device-resident cache length (a hint for attention kernels that size their
     // grid on the host; grows by the most a commit can add, exact again after prefill / generate read the length)
     int L_upper = 0;
@@ -186,7 +195,8 @@ struct ProfScope {
         }
     }
 };
-// `skip_mask` (MEDUSA_DEBUG_SKIP, a bit per category) drops launches: a timing aid to read a kernel class's
+#ifdef MEDUSA_TIMING_AIDS
+// Timing-aid builds only: `skip_mask` (MEDUSA_DEBUG_SKIP, a bit per category) drops launches, to read a kernel class's
 // cost inside the running pipeline; results are meaningless while it is set.
 #define PROF(c, cat, nk, stmt)                      \
     do {                                            \
@@ -195,6 +205,13 @@ struct ProfScope {
             stmt;                                   \
         }                                           \
     } while (0)
+#else
+#define PROF(c, cat, nk, stmt)               \
+    do {                                     \
+        ProfScope ps_((c), (cat), (nk));     \
+        stmt;                                \
+    } while (0)
+#endif
 
 #define TRY(expr)                          \
     do {                                   \
@@ -214,8 +231,13 @@ int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v
         // is not: it fills the SM's shared and tensor memory, so the projection that follows cannot stream its first
         // weight tiles while the attention runs (measured at 7B width up to 3860 keys).
         if (c->attn_mode == 2 || (c->attn_mode == 0 && !in_step && L_hint >= ATTN_TC_MIN_L))
+        {
+            const int wh = c->withhold == 2 ? 1 : 0;
+            if (wh) c->withhold = 0;
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_tc(q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse, c->flash_ws,
-                                                                  T, m.n_heads, c->Hkv, m.L_max, L_hint, c->d_state + ST_STATUS, c->stream));
+                                                                  T, m.n_heads, c->Hkv, m.L_max, L_hint, c->d_state + ST_STATUS, c->stream,
+                                                                  c->spin_limit, wh));
+        }
         else
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_flash(q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse,
                                                                      c->flash_ws, T, m.n_heads, c->Hkv, m.L_max, L_hint, c->stream));
@@ -243,8 +265,10 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
         if (!whole_tiles && (size_t)pd->n_max * plane_stride > c->part_elems)
             return fail(c, MEDUSA_ERR_SHAPE, "projection needs %d partial planes, more than the workspace holds", pd->n_max);
         cudaError_t e = cudaSuccess;
+        const int wh = c->withhold == 1 ? 1 : 0;
+        if (wh) c->withhold = 0;
         PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, n_seg, seg_cols, K, *pd, P, ldy, T, row0, c->d_state + ST_STATUS,
-                                               c->stream, seg0_cols));
+                                               c->stream, seg0_cols, c->spin_limit, wh));
         if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "tensor-core GEMM launch failed: %s", cudaGetErrorString(e));
         return MEDUSA_OK;
     }
@@ -285,6 +309,15 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
         // x += down-projection of the previous layer;  xn = RMSNorm(x)
         PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd_prev, w[0], m.rms_eps, c->xn, c->lo(c->xn, d), nullptr, T,
                                                    d, s));
+        if (c->tap_layer >= 0) {
+            const size_t planes = dt == MEDUSA_BF16 ? 2 : 1;
+            if (l == c->tap_layer)
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_in, c->x, (size_t)TREE_ROWS * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+            if (l == c->tap_layer + 1) {
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)TREE_ROWS * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->xn, planes * TREE_ROWS * d * c->esz, cudaMemcpyDeviceToDevice, s));
+            }
+        }
         const void *wqkv[3] = {w[1], w[2], w[3]};
         if (Hkv == H || !c->use_tc || (HD % 128 == 0 && HkvD % 128 == 0)) {
             // one launch for [q | k | v]; with grouped-query attention the k and v matrices are narrower than q
@@ -301,6 +334,9 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
         }
         MEDUSA_LAUNCH_CHECK(c);
         TRY(attention(c, c->q, tk, tv, kc, vc, cache_len, mask, c->att, c->lo(c->att, HD), nullptr, T, c->L_upper, true));
+        if (l == c->tap_layer)
+            MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_att, c->att, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)TREE_ROWS * HD * c->esz,
+                                           cudaMemcpyDeviceToDevice, s));
         const void *wo[1] = {w[4]};
         TRY(project(c, c->att, &c->map_att, wo, wm ? wm + 3 : nullptr, 1, d, HD, c->part, (size_t)TREE_ROWS * d, d, T, 0, false, &pd));
         // x += attention output projection;  xn = RMSNorm(x)
@@ -314,6 +350,11 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
     }
     PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd_prev, c->w.final_norm, m.rms_eps, c->hidden,
                                                c->lo(c->hidden, d), c->hidden_f32, T, d, s));
+    if (c->tap_layer >= 0 && c->tap_layer == m.n_layers - 1) {
+        MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)TREE_ROWS * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+        MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->hidden, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)TREE_ROWS * d * c->esz,
+                                       cudaMemcpyDeviceToDevice, s));
+    }
     MEDUSA_LAUNCH_CHECK(c);
     // LM head straight into the logits buffer: whole tiles, one plane
     const void *wl[1] = {c->w.lm_head};
@@ -334,6 +375,8 @@ int32_t check_ready(medusa_ctx *c, bool need_tree, bool need_weights)
 }  // namespace
 
 // ============================================================================ lifetime
+
+static void drop_step_graphs(medusa_ctx *c);
 
 extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc, int32_t device, void *stream)
 {
@@ -366,8 +409,8 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
         else { c->stream = nullptr; (void)cudaGetLastError(); }
     }
     c->esz = m.dtype == MEDUSA_BF16 ? 2 : 4;
-    if (const char *sk = getenv("MEDUSA_DEBUG_SKIP")) c->skip_mask = (unsigned)atoi(sk);
-    if (const char *sg = getenv("MEDUSA_STEP_GRAPH")) c->step_graphs_on = atoi(sg) != 0;
+    if (const char *sk = tuning_env("MEDUSA_DEBUG_SKIP")) c->skip_mask = (unsigned)atoi(sk);
+    if (const char *sg = tuning_env("MEDUSA_STEP_GRAPH")) c->step_graphs_on = atoi(sg) != 0;
     *out = c;
     MEDUSA_CUDA(c, cudaSetDevice(device));
     c->Hkv = m.n_kv_heads > 0 ? m.n_kv_heads : m.n_heads;
@@ -407,11 +450,15 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     TRY(dev_alloc_bytes(c, &c->node_part, R * NODE_STAT_SLICES * NODE_PART_BYTES));
     TRY(dev_alloc(c, &c->gumbel_dev, V));
     TRY(dev_alloc_bytes(c, &c->topk_scratch, topk_scratch_bytes(m.n_medusa > 0 ? m.n_medusa : 1)));
-    if (m.dtype == MEDUSA_BF16 && m.head_dim == 128 && getenv("MEDUSA_FORCE_SIMT_ATTENTION") == nullptr)
+    TRY(dev_alloc(c, &c->tap_x_in, R * d));
+    TRY(dev_alloc(c, &c->tap_x_out, R * d));
+    TRY(dev_alloc_bytes(c, &c->tap_att, planes * R * HD * c->esz));
+    TRY(dev_alloc_bytes(c, &c->tap_xn_out, planes * R * d * c->esz));
+    if (m.dtype == MEDUSA_BF16 && m.head_dim == 128 && tuning_env("MEDUSA_FORCE_SIMT_ATTENTION") == nullptr)
         TRY(dev_alloc_bytes(c, &c->flash_ws, tree_attention_flash_workspace_bytes(m.n_heads)));
-    if (const char *e = getenv("MEDUSA_ATTENTION"))
+    if (const char *e = tuning_env("MEDUSA_ATTENTION"))
         c->attn_mode = strcmp(e, "tcgen05") == 0 ? 2 : (strcmp(e, "mma_sync") == 0 ? 1 : 0);
-    c->use_tc = m.dtype == MEDUSA_BF16 && getenv("MEDUSA_FORCE_SIMT_GEMM") == nullptr && !(d % 8 || HD % 8 || HkvD % 8 || F % 8);
+    c->use_tc = m.dtype == MEDUSA_BF16 && tuning_env("MEDUSA_FORCE_SIMT_GEMM") == nullptr && !(d % 8 || HD % 8 || HkvD % 8 || F % 8);
     {
         // partial planes: for each projection, its width times the most pieces any of its tiles is cut into
         const size_t qkv_ld = HD + 2 * HkvD;
@@ -455,14 +502,6 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     return MEDUSA_OK;
 }
 
-// Drops every captured step graph: called when something a graph has baked in changes (tree, weights).
-static void drop_step_graphs(medusa_ctx *c)
-{
-    for (auto &g : c->step_graphs) cudaGraphExecDestroy(g.exec);
-    c->step_graphs.clear();
-    c->have_last_key = false;
-}
-
 extern "C" int32_t medusa_destroy(medusa_ctx *c)
 {
     if (!c) return MEDUSA_ERR_INVALID_ARG;
@@ -490,24 +529,91 @@ extern "C" int32_t medusa_device_status(medusa_ctx *c)
     return st;
 }
 
+// Drops every captured step graph: called when something a graph has baked in changes (tree, weights).
+static void drop_step_graphs(medusa_ctx *c)
+{
+    for (auto &g : c->step_graphs) cudaGraphExecDestroy(g.exec);
+    c->step_graphs.clear();
+    c->have_last_key = false;
+}
+
+// Context-owned buffer `which` and its size in bytes (0 bytes: not allocated yet).
+static const void *workspace_view(medusa_ctx *c, int32_t which, size_t *bytes)
+{
+    const medusa_model_desc &m = c->m;
+    const size_t R = TREE_ROWS, d = m.d, V = m.vocab, K = m.n_medusa ? m.n_medusa : 1, HD = (size_t)m.n_heads * m.head_dim;
+    const size_t HkvD = (size_t)c->Hkv * m.head_dim, planes = m.dtype == MEDUSA_BF16 ? 2 : 1;
+    const size_t cache_bytes = (size_t)m.n_layers * HkvD * m.L_max * c->esz, tree_bytes = (size_t)m.n_layers * R * HkvD * c->esz;
+    const void *p = nullptr;
+    size_t n = 0;
+    switch (which) {
+    case MEDUSA_WS_LOGITS: p = c->logits; n = R * V * sizeof(float); break;
+    case MEDUSA_WS_HIDDEN: p = c->hidden_f32; n = R * d * sizeof(float); break;
+    case MEDUSA_WS_TREE_K: p = c->tree_k; n = tree_bytes; break;
+    case MEDUSA_WS_TREE_V: p = c->tree_v; n = tree_bytes; break;
+    case MEDUSA_WS_K_CACHE: p = c->k_cache; n = cache_bytes; break;
+    case MEDUSA_WS_V_CACHE: p = c->v_cache; n = cache_bytes; break;
+    case MEDUSA_WS_HEAD_LOGITS: p = c->head_logits; n = K * V * sizeof(float); break;
+    case MEDUSA_WS_TOPK_IDX: p = c->topk_idx; n = K * R * sizeof(int32_t); break;
+    case MEDUSA_WS_TREE_TOK: p = c->tree_tok; n = R * sizeof(int32_t); break;
+    case MEDUSA_WS_ACC_NODES: p = c->acc_nodes; n = R * sizeof(int32_t); break;
+    case MEDUSA_WS_STATE: p = c->d_state; n = ST_WORDS * sizeof(int32_t); break;
+    case MEDUSA_WS_H_LAST: p = c->h_last; n = d * sizeof(float); break;
+    case MEDUSA_WS_EMITTED: p = c->emitted; n = R * sizeof(int32_t); break;
+    case MEDUSA_WS_TAP_X_IN: p = c->tap_x_in; n = R * d * sizeof(float); break;
+    case MEDUSA_WS_TAP_X_OUT: p = c->tap_x_out; n = R * d * sizeof(float); break;
+    case MEDUSA_WS_TAP_ATT: p = c->tap_att; n = planes * R * HD * c->esz; break;
+    case MEDUSA_WS_TAP_XN_OUT: p = c->tap_xn_out; n = planes * R * d * c->esz; break;
+    default: break;
+    }
+    if (bytes) *bytes = p ? n : 0;
+    return p;
+}
+
 extern "C" const void *medusa_workspace_ptr(medusa_ctx *c, int32_t which)
 {
-    if (!c) return nullptr;
-    switch (which) {
-    case MEDUSA_WS_LOGITS: return c->logits;
-    case MEDUSA_WS_HIDDEN: return c->hidden_f32;
-    case MEDUSA_WS_TREE_K: return c->tree_k;
-    case MEDUSA_WS_TREE_V: return c->tree_v;
-    case MEDUSA_WS_K_CACHE: return c->k_cache;
-    case MEDUSA_WS_V_CACHE: return c->v_cache;
-    case MEDUSA_WS_HEAD_LOGITS: return c->head_logits;
-    case MEDUSA_WS_TOPK_IDX: return c->topk_idx;
-    case MEDUSA_WS_TREE_TOK: return c->tree_tok;
-    case MEDUSA_WS_ACC_NODES: return c->acc_nodes;
-    case MEDUSA_WS_STATE: return c->d_state;
-    case MEDUSA_WS_H_LAST: return c->h_last;
-    case MEDUSA_WS_EMITTED: return c->emitted;
-    default: return nullptr;
+    return c ? workspace_view(c, which, nullptr) : nullptr;
+}
+
+extern "C" int32_t medusa_set_option(medusa_ctx *c, int32_t option, int64_t value)
+{
+    if (!c) return MEDUSA_ERR_INVALID_ARG;
+    switch (option) {
+    case MEDUSA_OPT_STEP_GRAPHS:
+        c->step_graphs_on = value != 0;
+        if (!c->step_graphs_on) {
+            MEDUSA_CUDA(c, cudaSetDevice(c->device));
+            MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
+            drop_step_graphs(c);
+        }
+        return MEDUSA_OK;
+    case MEDUSA_OPT_ATTENTION_KERNEL:
+        if (value < 0 || value > 2) return fail(c, MEDUSA_ERR_INVALID_ARG, "attention kernel must be 0 (automatic), 1 (mma.sync) or 2 (tcgen05)");
+        c->attn_mode = (int)value;
+        return MEDUSA_OK;
+    case MEDUSA_OPT_ATTENTION_LENGTH_HINT:
+        c->attn_len_hint = value < 0 ? -1 : (value > c->m.L_max ? c->m.L_max : (int)value);
+        return MEDUSA_OK;
+    case MEDUSA_OPT_LAYER_TAP:
+        if (value >= c->m.n_layers) return fail(c, MEDUSA_ERR_INVALID_ARG, "layer tap %lld: the model has %d layers", (long long)value, c->m.n_layers);
+        MEDUSA_CUDA(c, cudaSetDevice(c->device));
+        MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
+        drop_step_graphs(c);  // captured steps have the old tap baked in
+        c->tap_layer = value < 0 ? -1 : (int)value;
+        return MEDUSA_OK;
+    case MEDUSA_OPT_SPIN_LIMIT:
+        if (value < 0 || value > 0x7fffffffLL) return fail(c, MEDUSA_ERR_INVALID_ARG, "spin limit out of range");
+        MEDUSA_CUDA(c, cudaSetDevice(c->device));
+        MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
+        drop_step_graphs(c);  // captured launches carry the old limit
+        c->spin_limit = (uint32_t)value;
+        return MEDUSA_OK;
+    case MEDUSA_OPT_WITHHOLD_LOAD:
+        if (value < 0 || value > 2) return fail(c, MEDUSA_ERR_INVALID_ARG, "withhold: 0 (off), 1 (next tensor-core GEMM) or 2 (next tcgen05 attention)");
+        c->withhold = (int)value;
+        return MEDUSA_OK;
+    default:
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "unknown option %d", option);
     }
 }
 
@@ -549,12 +655,30 @@ extern "C" int32_t medusa_get_profile(medusa_ctx *c, double *ms_host, int64_t *l
 extern "C" int32_t medusa_read_workspace(medusa_ctx *c, int32_t which, int64_t offset_bytes, void *dst_host, int64_t bytes)
 {
     if (!c || !dst_host || offset_bytes < 0 || bytes < 0) return MEDUSA_ERR_INVALID_ARG;
-    const char *p = (const char *)medusa_workspace_ptr(c, which);
+    size_t have = 0;
+    const char *p = (const char *)workspace_view(c, which, &have);
     if (!p) return fail(c, MEDUSA_ERR_STATE, "workspace buffer %d does not exist (yet)", which);
+    if ((uint64_t)offset_bytes + (uint64_t)bytes > have)
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_read_workspace: bytes [%lld, %lld) lie outside buffer %d of %zu bytes",
+                    (long long)offset_bytes, (long long)(offset_bytes + bytes), which, have);
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
     MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
     MEDUSA_CUDA(c, cudaMemcpy(dst_host, p + offset_bytes, (size_t)bytes, cudaMemcpyDeviceToHost));
     return MEDUSA_OK;
+}
+
+// Measurement aid (no counterpart in the method): enqueues a kernel that reads `bytes` bytes of `buf` with 16-byte
+// streaming loads and writes nothing but a few floats to `sink`.
+extern "C" int32_t medusa_stream_read(const void *buf, int64_t bytes, float *sink, int32_t sink_floats, void *stream)
+{
+    if (!buf || !sink || bytes < 16 || sink_floats < 1 || ((uintptr_t)buf & 15u)) return MEDUSA_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return MEDUSA_ERR_CUDA;
+    int blocks = sms * 4;
+    if (blocks > sink_floats) blocks = sink_floats;
+    launch_stream_read(buf, (long long)bytes, sink, blocks, (cudaStream_t)stream);
+    return cudaGetLastError() == cudaSuccess ? MEDUSA_OK : MEDUSA_ERR_CUDA;
 }
 
 // ============================================================================ a0: tree
@@ -655,8 +779,10 @@ extern "C" int32_t medusa_tree_attention(medusa_ctx *c, const void *q, const voi
         kk = c->rot_k;
     }
     MEDUSA_LAUNCH_CHECK(c);
-    // the cache length lives on the device here: size the grid for the full capacity
-    return attention(c, qq, kk, v_new, k_cache, v_cache, cache_len, c->d_mask, out, nullptr, lse, T, m.L_max, false);
+    // the cache length lives on the device here: the kernel choice and the tcgen05 kernel's grid follow the caller's
+    // bound (MEDUSA_OPT_ATTENTION_LENGTH_HINT), or the full capacity if none was given
+    const int hint = c->attn_len_hint < 0 || c->attn_len_hint > m.L_max ? m.L_max : c->attn_len_hint;
+    return attention(c, qq, kk, v_new, k_cache, v_cache, cache_len, c->d_mask, out, nullptr, lse, T, hint, false);
 }
 
 // ============================================================================ a7: acceptance
@@ -911,7 +1037,7 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
     // of the cache length, which a captured launch would freeze)
     bool graphed = false;
     cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
-    if (c->step_graphs_on && !c->prof && c->skip_mask == 0 && c->attn_mode != 2 &&
+    if (c->step_graphs_on && !c->prof && c->skip_mask == 0 && c->attn_mode != 2 && c->withhold == 0 &&
         cudaStreamIsCapturing(c->stream, &capturing) == cudaSuccess && capturing == cudaStreamCaptureStatusNone) {
         medusa_ctx::StepKey key;
         memset(&key, 0, sizeof key);

@@ -327,7 +327,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     const int h = blockIdx.x, sp = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 3, kh = warp >> 2;  // query-row group, key half
-    const int L = *a.cache_len;
+    // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
+    const int L = min(max(*a.cache_len, 0), a.L_max);
     const int nt = (L + BKEY - 1) / BKEY;
     if (nt <= a.rows_max_tiles && gridDim.y >= 2) {
         if (sp < 2)
@@ -346,12 +347,14 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
         tps = nt > 0 ? (nt + want - 1) / want : 1;
     }
     const int n_cache_splits = (nt + tps - 1) / tps;
-    const int n_active = n_cache_splits > 0 ? n_cache_splits : 1;
+    // never more ranges than the grid has rows: when the launch's fixed range size was chosen for a shorter cache than
+    // the one found here, the last range takes all the remaining tiles (slower, still complete)
+    const int n_active = min(n_cache_splits > 0 ? n_cache_splits : 1, (int)gridDim.y);
     if (sp >= n_active)
         return;
     const int tile0 = sp * tps;
-    const int tile1 = min(nt, tile0 + tps);
     const bool has_tree = sp == n_active - 1;
+    const int tile1 = has_tree ? nt : min(nt, tile0 + tps);
     const int n_tiles = (tile1 - tile0) + (has_tree ? 1 : 0);
     const size_t HD = (size_t)a.H * D, HkvD = (size_t)a.Hkv * D;
     const int hk = h / (a.H / a.Hkv);
@@ -688,9 +691,11 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
 // Caches of up to this many 64-key tiles run in row-split mode (MEDUSA_ATTN_ROWS_MAX_TILES overrides, 0 = never).
 static int rows_mode_max_tiles()
 {
-    static const int v = getenv("MEDUSA_ATTN_ROWS_MAX_TILES") ? atoi(getenv("MEDUSA_ATTN_ROWS_MAX_TILES")) : 8;
+    static const int v = tuning_env("MEDUSA_ATTN_ROWS_MAX_TILES") ? atoi(tuning_env("MEDUSA_ATTN_ROWS_MAX_TILES")) : 8;
     return v;
 }
+
+static bool g_flash_attr_set[64] = {};  // devices on which the kernel's shared-memory limit has been raised
 
 size_t tree_attention_flash_workspace_bytes(int H)
 {
@@ -702,12 +707,10 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
                                         int L_hint, cudaStream_t s)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (first_use_on_current_device(g_flash_attr_set)) {
         cudaError_t e = cudaFuncSetAttribute(tree_attention_flash_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess)
             return e;
-        attr_set = true;
     }
     // One CTA per SM: the grid offers every head as many key ranges as fit one wave, the kernel uses the number
     // the true cache length asks for (the other CTAs leave at once).  L_hint is not needed for that.
@@ -715,7 +718,7 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
     int splits = 148 / H > 0 ? 148 / H : 1;
     if (splits > FLASH_MAX_SPLITS) splits = FLASH_MAX_SPLITS;
     int tps = 0;
-    if (const char *e = getenv("MEDUSA_ATTN_SPLITS")) {  // tuning aid: a fixed number of key ranges
+    if (const char *e = tuning_env("MEDUSA_ATTN_SPLITS")) {  // tuning aid: a fixed number of key ranges
         const int want = atoi(e);
         if (want > 0) {
             const int nt = ((L_hint < 0 || L_hint > L_max ? L_max : L_hint) + BKEY - 1) / BKEY;

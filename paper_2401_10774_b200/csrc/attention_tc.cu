@@ -45,7 +45,6 @@ constexpr int K_BYTES = 2 * KSUB_BYTES;
 constexpr int STAGE_BYTES = 2 * K_BYTES; // K then V
 constexpr int TAIL_BYTES = 4096;         // barriers and exchange buffers (struct Smem)
 constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + TAIL_BYTES;
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t O_COL = 256, P_COL = 384, Q_COL = 448;  // S0: 0..127, S1: 128..255, O': 256..383, P: 384..447, Q: 448..511
@@ -84,10 +83,10 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait.  Once any wait of the CTA has expired (`*failed`), every later wait returns immediately.
-__device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, volatile int *failed)
+__device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, volatile int *failed, uint32_t limit)
 {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\t"
                      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -242,6 +241,8 @@ struct Args {
     int32_t *status;                 // device status word
     int T, H, L_max, tiles_per_split;
     int Hkv;                         // key/value heads; query head h reads key/value head h / (H / Hkv)
+    uint32_t spin_limit;             // polls before a bounded wait gives up
+    int withhold;                    // test hook: CTA (0, 0)'s producer delivers no tile, so its consumers' waits expire
 };
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -253,15 +254,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
     Smem *sm = (Smem *)(ring + STAGES * STAGE_BYTES);
     const int h = blockIdx.x, sp = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int L = *a.cache_len;
+    const int L = min(max(*a.cache_len, 0), a.L_max);  // a length outside [0, L_max] would index past the caches
     const int nt = (L + BKEY - 1) / BKEY;
     const int n_cache_splits = (nt + a.tiles_per_split - 1) / a.tiles_per_split;
-    const int n_active = n_cache_splits > 0 ? n_cache_splits : 1;
+    // the range size was chosen on the host from an upper bound of the length; should the cache be longer than that,
+    // the grid's last row takes all the remaining tiles (slower, still complete)
+    const int n_active = min(n_cache_splits > 0 ? n_cache_splits : 1, (int)gridDim.y);
     if (sp >= n_active)
         return;
     const int tile0 = sp * a.tiles_per_split;
-    const int tile1 = min(nt, tile0 + a.tiles_per_split);
     const bool has_tree = sp == n_active - 1;
+    const int tile1 = has_tree ? nt : min(nt, tile0 + a.tiles_per_split);
     const int n_tiles = (tile1 - tile0) + (has_tree ? 1 : 0);  // >= 1
     const size_t HD = (size_t)a.H * D;
 
@@ -325,11 +328,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
         // rows = head * L_max + key); the ragged last cache tile and the tree's own keys by 16-byte asynchronous
         // copies with zero fill, so that no row beyond the cache length is ever read.
         const int hk = h / (a.H / a.Hkv);
-        for (int i = 0; i < n_tiles; ++i) {
+        const int n_deliver = a.withhold && h == 0 && sp == 0 ? 0 : n_tiles;
+        for (int i = 0; i < n_deliver; ++i) {
             const int st = i % STAGES;
             uint8_t *stage = ring + st * STAGE_BYTES;
             if (i >= STAGES)
-                mbar_wait(&sm->kv_empty[st], ((i / STAGES) - 1) & 1, failed);
+                mbar_wait(&sm->kv_empty[st], ((i / STAGES) - 1) & 1, failed, a.spin_limit);
             const int ct = tile0 + i;
             if (ct < tile1 && (ct + 1) * BKEY <= L) {
                 if (lane == 0) {
@@ -375,11 +379,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
         // as long as it takes the tensor core at these shapes, so two threads issue side by side.
         const uint32_t leader = lane == 0 ? 1u : 0u;
         if (warp == 8) {
-            mbar_wait(&sm->q_full, 0, failed);  // Q sits in tensor memory
+            mbar_wait(&sm->q_full, 0, failed, a.spin_limit);  // Q sits in tensor memory
             for (int i = 0; i < n_tiles; ++i) {
-                mbar_wait(&sm->kv_full[i % STAGES], (i / STAGES) & 1, failed);
+                mbar_wait(&sm->kv_full[i % STAGES], (i / STAGES) & 1, failed, a.spin_limit);
                 if (i >= 2)
-                    mbar_wait(&sm->s_empty[i & 1], ((i >> 1) - 1) & 1, failed);
+                    mbar_wait(&sm->s_empty[i & 1], ((i >> 1) - 1) & 1, failed, a.spin_limit);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t dk = desc_kmajor(smem_u32(ring + (i % STAGES) * STAGE_BYTES));
                 const uint32_t td = tmem + (uint32_t)((i & 1) * BKEY);
@@ -392,9 +396,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
             }
         } else {
             for (int i = 0; i < n_tiles; ++i) {
-                mbar_wait(&sm->p_full, i & 1, failed);
+                mbar_wait(&sm->p_full, i & 1, failed, a.spin_limit);
                 if (i >= 1)
-                    mbar_wait(&sm->o_empty, (i - 1) & 1, failed);
+                    mbar_wait(&sm->o_empty, (i - 1) & 1, failed, a.spin_limit);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t dv = desc_mnmajor(smem_u32(ring + (i % STAGES) * STAGE_BYTES) + K_BYTES);
 #pragma unroll
@@ -409,7 +413,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
         // every MMA of both warps has retired before the accumulators are freed, also after an expired wait
         umma_commit(&sm->done, leader);
         const uint32_t addr = smem_u32(&sm->done);
-        for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        for (uint32_t it = 0; it < a.spin_limit; ++it) {
             uint32_t ok;
             asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                          : "=r"(ok) : "r"(addr) : "memory");
@@ -441,7 +445,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
             float c = 0.f;
             if (i < n_tiles) {
                 float s[32];
-                mbar_wait(&sm->s_full[i & 1], (i >> 1) & 1, failed);
+                mbar_wait(&sm->s_full[i & 1], (i >> 1) & 1, failed, a.spin_limit);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 tmem_ld32(tmem + lane_addr + (uint32_t)((i & 1) * BKEY + copy * 64 + hf * 32), s);
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -482,7 +486,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
                 }
                 l = l * c + (ps0 + ps1);
                 if (i >= 1)
-                    mbar_wait(&sm->p_empty, (i - 1) & 1, failed);  // the previous tile's P V has read P
+                    mbar_wait(&sm->p_empty, (i - 1) & 1, failed, a.spin_limit);  // the previous tile's P V has read P
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 tmem_st16(tmem + lane_addr + P_COL + (uint32_t)(copy * 32 + hf * 16), pk);
                 tmem_st_wait();
@@ -493,7 +497,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
             }
             if (i > 0) {
                 // o = o * 2^(m_old - m_new) + P V of tile i - 1 (its MMA ran while this tile's scores were processed)
-                mbar_wait(&sm->o_full, (i - 1) & 1, failed);
+                mbar_wait(&sm->o_full, (i - 1) & 1, failed, a.spin_limit);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
                 for (int q2 = 0; q2 < 2; ++q2) {
@@ -662,7 +666,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                      const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                      void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                     int L_hint, int32_t *status, cudaStream_t s)
+                                     int L_hint, int32_t *status, cudaStream_t s, uint32_t spin_limit, int withhold)
 {
     // TMA descriptors of the two caches ([Hkv * L_max rows][128 dims] bf16, boxes of 64 dims x 128 rows), encoded once
     // per distinct cache
@@ -681,12 +685,11 @@ cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const voi
     const TensorMap *mk = map_of(k_cache), *mv = map_of(v_cache);
     if (!mk || !mv)
         return cudaErrorInvalidValue;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};
+    if (first_use_on_current_device(attr_set)) {
         cudaError_t e = cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess)
             return e;
-        attr_set = true;
     }
     if (L_hint > L_max) L_hint = L_max;
     if (L_hint < 0) L_hint = 0;
@@ -697,7 +700,7 @@ cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const voi
     while (want * want < nt) ++want;
     const int one_wave = 148 / H > 0 ? 148 / H : 1;
     if (want > one_wave) want = one_wave;
-    if (const char *e = getenv("MEDUSA_ATTN_SPLITS")) want = atoi(e) > 0 ? atoi(e) : want;
+    if (const char *e = tuning_env("MEDUSA_ATTN_SPLITS")) want = atoi(e) > 0 ? atoi(e) : want;
     int tps = nt > 0 ? (nt + want - 1) / want : 1;
     if (tps < 1) tps = 1;
     int splits = nt > 0 ? (nt + tps - 1) / tps : 1;
@@ -714,6 +717,8 @@ cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const voi
     a.counters = (int *)(a.ws_ml + (size_t)H * MAX_SPLITS * 2 * BQ);
     a.status = status;
     a.T = T; a.H = H; a.Hkv = Hkv; a.L_max = L_max; a.tiles_per_split = tps;
+    a.spin_limit = spin_limit ? spin_limit : DEFAULT_SPIN_LIMIT;
+    a.withhold = withhold;
     launch_pdl(tree_attention_tc_kernel, dim3(H, splits), dim3(THREADS), (size_t)SMEM_BYTES, s, *(const CUtensorMap *)mk,
                *(const CUtensorMap *)mv, a);
     return cudaGetLastError();

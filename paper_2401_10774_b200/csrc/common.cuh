@@ -3,6 +3,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <cstdlib>
 
 #include "../../include/medusa.h"
 
@@ -17,6 +18,33 @@ enum { ST_CACHE_LEN = 0, ST_ROOT = 1, ST_BEST = 2, ST_ACCEPT_LEN = 3, ST_NEXT_RO
        ST_STATUS = 6, ST_STEPS = 7, ST_WORDS = 8 };
 
 using bf16 = __nv_bfloat16;
+
+// Environment switches for comparison runs (MEDUSA_GEMM_STAGES, MEDUSA_NO_PDL, MEDUSA_DEBUG_SKIP, ...) exist only in a
+// library built with -DMEDUSA_TIMING_AIDS; the default build reads nothing from its caller's environment.
+inline const char *tuning_env(const char *name)
+{
+#ifdef MEDUSA_TIMING_AIDS
+    return getenv(name);
+#else
+    (void)name;
+    return nullptr;
+#endif
+}
+
+// True the first time it is called with the calling thread's current device (function attributes such as the
+// dynamic shared-memory limit are per device, so each device sets them once).
+inline bool first_use_on_current_device(bool (&done)[64])
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return true;
+    if (done[dev])
+        return false;
+    done[dev] = true;
+    return true;
+}
+
+constexpr uint32_t DEFAULT_SPIN_LIMIT = 1u << 22;  // polls of a bounded device-side wait before it gives up
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }

@@ -43,7 +43,6 @@ constexpr int B_BYTES = BN * BK * 2;    // 8 KiB per plane
 constexpr int STAGE_BYTES = A_BYTES + 2 * B_BYTES;
 constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */; }
 constexpr int THREADS = 192;
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -59,11 +58,11 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// bounded wait: false if the phase did not complete within SPIN_LIMIT polls
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// bounded wait: false if the phase did not complete within `limit` polls
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t limit)
 {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\t"
                      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -246,7 +245,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             uint32_t ph = 1;
             bool waited = false;  // has this thread waited for the preceding kernel yet
             int pend_k[MAX_STAGES], pend_n = 0;
-            bool ok = true;
+            bool ok = !(a.withhold && blockIdx.x == 0);  // test hook: this CTA's loads are withheld, nothing is in flight
             while (ok && it.next(sg)) {
                 // the first weight matrix may have its own number of tiles (a wider q beside narrower k and v)
                 const int rest = sg.tile - a.seg0_tiles;
@@ -266,7 +265,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                                 tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], BN, &sm->full[p], pol_keep);
                             }
                         }
-                        if (sm->failed || !mbar_wait(&sm->empty[s], ph)) {
+                        if (sm->failed || !mbar_wait(&sm->empty[s], ph, a.spin_limit)) {
                             sm->failed = 1;
                             ok = false;
                             break;
@@ -288,7 +287,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     }
                 }
             }
-            if (!waited) {
+            if (!waited && ok) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 for (int p = 0; p < pend_n; ++p) {
                     uint8_t *st = tiles + p * STAGE_BYTES;
@@ -308,14 +307,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             bool ok = true;
             while (ok && it.next(sg)) {
                 const int b = j & 1;
-                if (j >= 2 && (sm->failed || !mbar_wait(&sm->acc_empty[b], ((j >> 1) - 1) & 1))) {
+                if (j >= 2 && (sm->failed || !mbar_wait(&sm->acc_empty[b], ((j >> 1) - 1) & 1, a.spin_limit))) {
                     sm->failed = 1;
                     break;
                 }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");  // the epilogue has drained this accumulator
                 const uint32_t tmem_d = tmem_base + (uint32_t)(b * UMMA_N);
                 for (int i = 0; i < sg.nkb; ++i) {
-                    if (sm->failed || !mbar_wait(&sm->full[st], ph)) {
+                    if (sm->failed || !mbar_wait(&sm->full[st], ph, a.spin_limit)) {
                         sm->failed = 1;
                         ok = false;
                         break;
@@ -346,7 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         int j = 0;
         while (it.next(sg)) {
             const int b = j & 1;
-            const bool ready = !sm->failed && mbar_wait(&sm->acc_full[b], (j >> 1) & 1);
+            const bool ready = !sm->failed && mbar_wait(&sm->acc_full[b], (j >> 1) & 1, a.spin_limit);
             if (!ready) {
                 sm->failed = 1;
                 break;
@@ -399,8 +398,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         if (threadIdx.x == 0) {
             atomicExch(a.status, MEDUSA_ERR_TIMEOUT);
             // loads already issued still write into this CTA's shared memory: wait (bounded) before exiting
-            for (int s = 0; s < STAGES; ++s)
-                (void)mbar_wait(&sm->full[s], 0);
+            if (!a.withhold)
+                for (int s = 0; s < STAGES; ++s)
+                    (void)mbar_wait(&sm->full[s], 0, a.spin_limit);
         }
         __syncthreads();
     }
@@ -451,7 +451,7 @@ bool make_act_map(TensorMap *out, const void *X_planes, int K) { return make_ten
 // CTAs resident per SM and TMA ring depth; MEDUSA_GEMM_CTAS_PER_SM / MEDUSA_GEMM_STAGES override for tuning
 static int env_int(const char *name, int dflt, int lo, int hi)
 {
-    const char *v = getenv(name);
+    const char *v = tuning_env(name);
     if (!v) return dflt;
     int x = atoi(v);
     return x < lo ? lo : (x > hi ? hi : x);
@@ -500,15 +500,14 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
 
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols)
+                           int seg0_cols, uint32_t spin_limit, int withhold)
 {
     if (seg0_cols <= 0) seg0_cols = seg_cols;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};
+    if (first_use_on_current_device(attr_set)) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(gemm_tc_stages()));
         if (e != cudaSuccess)
             return e;
-        attr_set = true;
     }
     GemmTcArgs a;
     a.P = P;
@@ -526,6 +525,8 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     a.row0 = row0;
     a.status = status;
     a.stages = gemm_tc_stages();
+    a.spin_limit = spin_limit ? spin_limit : DEFAULT_SPIN_LIMIT;
+    a.withhold = withhold;
     const CUtensorMap *w0 = (const CUtensorMap *)mapW[0];
     const CUtensorMap *w1 = (const CUtensorMap *)mapW[n_seg > 1 ? 1 : 0];
     const CUtensorMap *w2 = (const CUtensorMap *)mapW[n_seg > 2 ? 2 : 0];
@@ -536,7 +537,7 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = getenv("MEDUSA_NO_PDL") ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed = tuning_env("MEDUSA_NO_PDL") ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);

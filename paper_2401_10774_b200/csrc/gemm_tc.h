@@ -51,6 +51,8 @@ struct GemmTcArgs {
     int T, row0;             // token rows [row0, T) are stored
     int32_t *status;         // device status word (set to MEDUSA_ERR_TIMEOUT if a bounded wait expires)
     int stages;              // depth of the TMA ring
+    uint32_t spin_limit;     // polls before a bounded wait gives up
+    int withhold;            // test hook: CTA 0's producer issues no load at all, so its consumers' waits expire
 };
 
 // W: [N][K] bf16 row-major
@@ -66,6 +68,6 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
 // P[piece][t][first column of segment seg + n] = partial sums over k of (X_hi + X_lo)[t][k] * W_seg[n][k], t in [row0, T)
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols = 0);
+                           int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0);
 
 }  // namespace medusa

@@ -38,6 +38,9 @@ void launch_rope_apply(int dtype, const void *in, const float2 *cs, void *out, i
 void launch_silu_mul(int dtype, const float *gate_up, const PlaneDesc &pd, void *act, void *act_lo, int T,
                      int F, cudaStream_t s);
 
+// sums `bytes` bytes with 16-byte streaming loads (a pure DRAM read stream); sink: >= blocks floats
+void launch_stream_read(const void *buf, long long bytes, float *sink, int blocks, cudaStream_t s);
+
 // ---- attention.cu ----
 // q,out: [T][H][D], k_new,v_new: [T][Hkv][D] (already rotated); caches [Hkv][L_max][D]; mask [T]; lse nullable [T][H];
 // out_lo (nullable): second plane of the split output.  Hkv divides H: query head h reads key/value head h / (H / Hkv)
@@ -61,7 +64,7 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                      const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                      void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                     int L_hint, int32_t *status, cudaStream_t s);
+                                     int L_hint, int32_t *status, cudaStream_t s, uint32_t spin_limit = 0, int withhold = 0);
 
 // ---- heads.cu ----
 // x_k = h + SiLU(W1_k h) -> float [K][d];  h: float if h_is_f32 else the model dtype

@@ -21,10 +21,14 @@ __device__ __forceinline__ void pdl_enter()
     pdl_wait();
 }
 
-// MEDUSA_NO_PDL=1 launches every kernel fully serialised (for comparison runs)
+// MEDUSA_NO_PDL=1 launches every kernel fully serialised (comparison runs; builds with -DMEDUSA_TIMING_AIDS only)
 inline bool pdl_enabled()
 {
+#ifdef MEDUSA_TIMING_AIDS
     static const bool on = getenv("MEDUSA_NO_PDL") == nullptr;
+#else
+    static const bool on = true;
+#endif
     return on;
 }
 

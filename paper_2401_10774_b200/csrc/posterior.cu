@@ -340,8 +340,11 @@ __global__ void __launch_bounds__(256) commit_finalize_kernel(CommitArgs a)
     if (threadIdx.x == 0) {
         *a.n_emitted = n;
         *a.cache_len = L + n;
+        // The next step's root is the successor of the last COMMITTED token.  When max_commit cut the accepted path
+        // short (n < 1 + accept_len) that successor is the path's next node, which was already accepted; otherwise it
+        // is the token chosen after the whole path.
         if (a.root_out && a.next_root)
-            *a.root_out = *a.next_root;
+            *a.root_out = n > 0 && n < 1 + *a.accept_len ? a.tree_tok[a.acc_nodes[n]] : *a.next_root;
     }
 }
 

@@ -457,4 +457,34 @@ __global__ void iota_kernel(int32_t *p, int n)
 }
 void launch_iota(int32_t *p, int n, cudaStream_t s) { launch_pdl(iota_kernel, dim3((n + 63) / 64), dim3(64), 0, s, p, n); }
 
+// ---------------------------------------------------------------------------------------- read-only streaming probe
+// Sums a buffer with 16-byte loads, eight in flight per thread, and writes one float per block: nothing but a DRAM
+// read stream (the denominator for kernels that, like the projections and the attention, read far more than they write).
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4 *__restrict__ p, long long n16, float *sink)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t acc = 0;
+    for (; i + 7 * stride < n16; i += 8 * stride) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            v[u] = __ldcs(p + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            acc += v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+    }
+    for (; i < n16; i += stride) {
+        const uint4 v = __ldcs(p + i);
+        acc += v.x ^ v.y ^ v.z ^ v.w;
+    }
+    acc = __reduce_add_sync(0xffffffffu, acc);
+    if ((threadIdx.x & 31) == 0 && acc == 0x9e3779b9u)  // practically never: keeps the loads alive
+        sink[blockIdx.x] = 1.0f;
+}
+void launch_stream_read(const void *buf, long long bytes, float *sink, int blocks, cudaStream_t s)
+{
+    stream_read_kernel<<<blocks, 512, 0, s>>>((const uint4 *)buf, bytes / 16, sink);
+}
+
 }  // namespace medusa

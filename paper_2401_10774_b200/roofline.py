@@ -82,3 +82,34 @@ def hbm_peak_gbs():
     if os.path.exists(p):
         return float(json.load(open(p))["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+# ---- DRAM traffic taken from profiler captures ----
+# A capture describes the kernel source it was taken from: the figure is reported only while the SHA-256 of that
+# source file still equals the one recorded with the capture, so a changed kernel never inherits an old number.
+# bytes = dram__bytes_read.sum + dram__bytes_write.sum per launch, the launch-weighted mean over one step's launches
+# (the four layer shapes captured on a 2-layer model of the same width: a layer's traffic does not depend on the
+# depth; the LM head's figure is its weights plus the logits).
+CAPTURED_TRAFFIC = {
+    # (kernel, model): (bytes per launch, source file, sha256 of that file at capture time)
+    ("gemm_tc_kernel", "7b"): (108.3e6, "csrc/gemm_tc.cu", "0" * 64),
+}
+
+
+def captured_traffic(kernel: str, model: str):
+    """-> (bytes per launch or None, note)"""
+    import hashlib
+    import os
+
+    rec = CAPTURED_TRAFFIC.get((kernel, model))
+    if rec is None:
+        return None, "no profiler capture of %s at the %s shape" % (kernel, model)
+    nbytes, rel, sha = rec
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), rel)
+    try:
+        now = hashlib.sha256(open(path, "rb").read()).hexdigest()
+    except OSError:
+        return None, "kernel source %s not found" % rel
+    if now != sha:
+        return None, "the profiler capture of %s is older than its source (%s changed since): not reported" % (kernel, rel)
+    return nbytes, "profiler capture of %s taken from the current %s" % (kernel, rel)

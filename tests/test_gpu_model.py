@@ -282,7 +282,7 @@ def test_tiny_fp32_typical_sampled_generate_matches_oracle(oracle):
 
 
 @pytest.mark.parametrize("mode", ["greedy", "typical_gumbel"])
-def test_step_graph_replay_matches_plain_launches(oracle, mode, monkeypatch):
+def test_step_graph_replay_matches_plain_launches(oracle, mode):
     # The library captures a decode step into a CUDA graph on the second use of a launch configuration.  The same
     # steps with the graphs switched off must leave bit-identical state behind, across a change of the attention
     # grid (the cache grows through several 64-key tiles) and with the host following the cache length without
@@ -296,9 +296,9 @@ def test_step_graph_replay_matches_plain_launches(oracle, mode, monkeypatch):
     noise = torch.from_numpy(I.gumbel_noise(steps, cfg["vocab"], 52)).cuda() if mode != "greedy" else None
     pinned = torch.zeros(2 * steps * 8, dtype=torch.int32).pin_memory()
     runs = []
-    for graphs in ("1", "0"):
-        monkeypatch.setenv("MEDUSA_STEP_GRAPH", graphs)
+    for graphs in (1, 0):
         ctx = U.make_ctx(cfg, "bf16", L_max, I.TREE_SPECS["sparse64_d4"])
+        ctx.set_option(B.OPT_STEP_GRAPHS, graphs)
         ctx.load_weights(U.dev_weights(w))
         ctx.prefill(prompt)
         lens = []
@@ -342,4 +342,26 @@ def test_bad_acceptance_mode_is_refused_and_leaves_the_step_graphs_on(oracle):
     torch.cuda.synchronize()
     info = ctx.step_graph_info()
     assert info["graphs"] == 1 and info["replays"] >= 3 and ctx.device_status() == 0
+    ctx.close()
+
+
+def test_decode_with_commit_budget_of_one_continues_the_same_stream(oracle):
+    """A caller that lets every step commit a single token (max_commit = 1) still walks the greedy token stream: after
+    a truncated commit the next root is the accepted path's next token, not the token after the whole path."""
+    torch, B, U = _gpu()
+    cfg = I.model_shape("tiny")
+    ctx, om, ot = _setup(oracle, cfg, "f32", "dense22", 128, seed=0, head_init="lm_copy")
+    prompt = I.make_prompt(32, cfg["vocab"], 1)
+    G = 40
+    plain = oracle.generate_plain(om, prompt, G, 128)["tokens"].tolist()
+    ctx.prefill(torch.from_numpy(prompt).cuda())
+    got, truncated = [], 0
+    for s in range(G):
+        ctx.decode_step(B.AcceptParams(mode=B.GREEDY), None, max_commit=1)
+        st = ctx.state()
+        assert st["n_emitted"] == 1 and st["cache_len"] == 32 + s + 1 and st["status"] == 0
+        got.append(int(ctx.read_workspace(B.WS_EMITTED, (1,), np.int32)[0]))
+        truncated += st["accept_len"] > 0
+    assert got == plain
+    assert truncated > 0, "the budget must actually have cut accepted paths short for this test to mean anything"
     ctx.close()

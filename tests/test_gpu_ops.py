@@ -41,12 +41,15 @@ ATT_CASES = [
 ]
 
 
-def _run_attention_case(oracle, case):
+def _run_attention_case(oracle, case, kernel=0, length_hint=None):
     torch, B, U = _gpu()
     name, dt, H, D, L, L_max, tree_name, rope = case[:8]
     Hkv = case[8] if len(case) > 8 else 0
     cfg = dict(n_layers=0, d=H * D, n_heads=H, n_kv_heads=Hkv, head_dim=D, ffn=8, vocab=8, n_medusa=5)
     ctx = U.make_ctx(cfg, dt, L_max, I.TREE_SPECS[tree_name])
+    ctx.set_option(B.OPT_ATTENTION_KERNEL, kernel)
+    if length_hint is not None:
+        ctx.set_option(B.OPT_ATTENTION_LENGTH_HINT, length_hint)
     t = ctx.tree
     seed = 20 if L <= 1024 else 21
     a = I.attention_inputs(t["T"], H, D, L, L_max, seed, dtype=dt, Hkv=Hkv)
@@ -81,10 +84,17 @@ TC_ATT_CASES = [c for c in ATT_CASES if c[1] == "bf16" and c[3] == 128] + [
 
 
 @pytest.mark.parametrize("case", TC_ATT_CASES, ids=[c[0] for c in TC_ATT_CASES])
-def test_tree_attention_parity_tcgen05_kernel(oracle, case, monkeypatch):
-    """The tcgen05/TMEM variant of the attention kernel (selected when the context is created) meets the same bar."""
-    monkeypatch.setenv("MEDUSA_ATTENTION", "tcgen05")
-    _run_attention_case(oracle, case)
+def test_tree_attention_parity_tcgen05_kernel(oracle, case):
+    """The tcgen05/TMEM variant of the attention kernel (selected with MEDUSA_OPT_ATTENTION_KERNEL) meets the same bar."""
+    _run_attention_case(oracle, case, kernel=2)
+
+
+@pytest.mark.parametrize("kernel", [1, 2], ids=["mma_sync", "tcgen05"])
+@pytest.mark.parametrize("hint", [0, 300, 2500])
+def test_tree_attention_length_hint_is_only_a_hint(oracle, kernel, hint):
+    """A host-side length bound that is too small (or exact) changes the launch, never the result."""
+    _run_attention_case(oracle, ("bf16_gqa_H16_kv4_L2500", "bf16", 16, 128, 2500, 2560, "sparse64_d4", True, 4),
+                        kernel=kernel, length_hint=hint)
 
 
 def _random_tree_paths(g, depth, target):
@@ -102,13 +112,12 @@ def _random_tree_paths(g, depth, target):
 
 @pytest.mark.parametrize("kernel", ["default", "tcgen05"])
 @pytest.mark.parametrize("dt,D", [("bf16", 128), ("f32", 64)])
-def test_tree_attention_random_trees(oracle, dt, D, kernel, monkeypatch):
+def test_tree_attention_random_trees(oracle, dt, D, kernel):
     """Irregular trees (any shape a caller may upload: chains, stars, lopsided ones, 2 to 64 nodes) at ragged cache
     lengths: the ancestor masks, positions and the tail tile must be right for every one of them."""
     if kernel == "tcgen05":
         if dt != "bf16":
             pytest.skip("the TMEM kernel exists for bf16, head dim 128")
-        monkeypatch.setenv("MEDUSA_ATTENTION", "tcgen05")
     torch, B, U = _gpu()
     g = I.rng(61, "random-attention-trees")
     H = 3
@@ -121,6 +130,7 @@ def test_tree_attention_random_trees(oracle, dt, D, kernel, monkeypatch):
         L_max = 256
         cfg = dict(n_layers=0, d=H * D, n_heads=H, head_dim=D, ffn=8, vocab=8, n_medusa=5)
         ctx = U.make_ctx(cfg, dt, L_max, paths=paths)
+        ctx.set_option(B.OPT_ATTENTION_KERNEL, 2 if kernel == "tcgen05" else 0)
         T = ctx.tree["T"]
         a = I.attention_inputs(T, H, D, L, L_max, 70 + trial, dtype=dt)
         dev = {k: U.to_dev(v) for k, v in a.items()}

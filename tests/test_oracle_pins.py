@@ -621,3 +621,36 @@ def test_typical_generate_accepts_more_and_is_deterministic(oracle):
     assert a["tokens"].tolist() == b["tokens"].tolist()
     assert np.all(a["emitted_per_step"] >= 1) and np.all(a["emitted_per_step"] <= 3)
     assert a["steps"] <= gr["steps"]
+
+
+# ----------------------------------------------------------------------------- single-layer entry (layer-by-layer parity checks)
+
+def test_layer_entry_composes_to_the_tree_pass_and_bf16_storage_rounding(oracle):
+    """ora_layer runs the same block the pass runs: chaining it over the layers from the embedding rows, then the closing
+    norm and LM head, reproduces ora_tree_pass bit for bit.  With kv_bf16 the tree keys/values are the unrounded ones
+    rounded to bfloat16 (checked against numpy's own float32 -> bfloat16 rounding)."""
+    cfg = I.model_shape("tiny", n_kv_heads=2)
+    w = I.make_weights(cfg, seed=3, dtype="f32", gain_std=0.1)
+    om = oracle.Model(cfg, w)
+    t = oracle.build_tree_buffers(oracle.default_tree_paths((2, 2), 7))
+    L_max, L = 24, 9
+    g = I.rng(77, "layer-entry")
+    kc = g.standard_normal(om.cache_shape(L_max))
+    vc = g.standard_normal(om.cache_shape(L_max))
+    tok = g.integers(0, cfg["vocab"], size=t["T"]).astype(np.int32)
+    ref = oracle.tree_pass(om, tok, t, L, kc, vc)
+    x = I.as_f32(w["embed"])[tok].astype(np.float64)
+    for l in range(cfg["n_layers"]):
+        r = oracle.layer(om, l, x, t, L, np.ascontiguousarray(kc[l]), np.ascontiguousarray(vc[l]))
+        assert np.array_equal(r["tree_k"], ref["tree_k"][l]) and np.array_equal(r["tree_v"], ref["tree_v"][l])
+        rb = oracle.layer(om, l, x, t, L, np.ascontiguousarray(kc[l]), np.ascontiguousarray(vc[l]), kv_bf16=True)
+        for name in ("tree_k", "tree_v"):
+            want = I.bf16_bits_to_f32(I.to_bf16_bits(r[name].astype(np.float32)))
+            assert np.array_equal(rb[name], want.astype(np.float64))
+        assert np.abs(rb["x_out"] - r["x_out"]).max() < 1e-2  # storage rounding moves the output only slightly
+        x = r["x_out"]
+    fin = oracle.final_norm_lm_head(om, x=x)
+    assert np.array_equal(fin["hidden"], ref["hidden"]) and np.array_equal(fin["logits"], ref["logits"])
+    # the LM head alone on a given hidden state
+    alone = oracle.final_norm_lm_head(om, hidden_in=ref["hidden"])
+    assert np.array_equal(alone["logits"], ref["logits"])

@@ -14,14 +14,21 @@ pytestmark = pytest.mark.gpu
 TOL_ATTN_BF16 = 2e-2  # the tolerance the other attention parity tests use (max abs, bf16 outputs)
 
 
-@pytest.mark.parametrize("L", [0, 300, 1000])
-def test_static_entry_matches_context_entry_twice(L):
+# (cache length, heads, capacity, length hint given to the call): the hint sizes the launch and may be exact, absent
+# (-1: the capacity is assumed) or too small (the result must not change); 2000 and 3000 keys use several key ranges
+# per head, i.e. the fixed scratch array really carries partial results between CTAs
+CASES = [(0, 8, 1024, 0), (300, 8, 1024, 300), (1000, 8, 1024, 1000), (1000, 8, 1024, -1), (2000, 32, 2048, 2000),
+         (2000, 32, 2048, 100), (3000, 64, 3072, -1)]
+
+
+@pytest.mark.parametrize("L,H,L_max,hint", CASES)
+def test_static_entry_matches_context_entry_twice(oracle, L, H, L_max, hint):
     import torch
     from paper_2401_10774_b200 import binding as B
     from tests import gpu_util as U
 
     assert torch.cuda.is_available(), "this test needs a CUDA device"
-    H, D, L_max = 8, 128, 1024
+    D = 128
     cfg = dict(n_layers=0, d=H * D, n_heads=H, head_dim=D, ffn=8, vocab=8, n_medusa=4)
     ctx = U.make_ctx(cfg, "bf16", L_max, I.TREE_SPECS["sparse64_d4"])
     t = ctx.tree
@@ -39,9 +46,17 @@ def test_static_entry_matches_context_entry_twice(L):
         out = torch.full((T, H, D), float("nan"), dtype=torch.bfloat16, device="cuda")
         lse = torch.full((T, H), float("nan"), dtype=torch.float32, device="cuda")
         B.tree_attention_static(dev["q"], dev["k_new"], dev["v_new"], dev["k_cache"], dev["v_cache"], cache_len, mask,
-                                T, H, L_max, L, out, lse)
+                                T, H, L_max, hint, out, lse)
         torch.cuda.synchronize()
         outs.append((out, lse))
+    # against the oracle too (same bar as the other attention parity tests)
+    ot = oracle.build_tree_buffers(oracle.default_tree_paths(**I.TREE_SPECS["sparse64_d4"]))
+    o_ref, o_lse = oracle.tree_attention(*(I.as_f32(a[k]) for k in ("q", "k_new", "v_new", "k_cache", "v_cache")), L,
+                                         ot["mask"], ot["pos"], apply_rope=False)
+    for out, lse in outs:
+        err = np.abs(U.to_host_f32(out) - o_ref).max()
+        assert err <= TOL_ATTN_BF16, "max |err| %.3g vs the oracle" % err
+        assert np.abs(U.to_host_f32(lse) - o_lse).max() <= 5e-2
     for out, lse in outs:
         err = (out.float() - ref.float()).abs().max().item()
         assert err <= TOL_ATTN_BF16, "max |err| %.3g vs the context entry point" % err
