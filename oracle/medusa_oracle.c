@@ -552,7 +552,9 @@ void ora_tree_attention(const float *q, const float *k_new, const float *v_new, 
 
 typedef struct {
     int32_t n_layers, d, n_heads, head_dim, ffn, vocab, n_medusa, wdtype; /* wdtype 0 f32, 1 bf16 bits */
-    int32_t n_kv_heads, pad_;  /* key/value heads (grouped-query attention); 0 means n_heads */
+    int32_t n_kv_heads;  /* key/value heads (grouped-query attention); 0 means n_heads */
+    int32_t kv_bf16;     /* != 0: every pass holds its tree keys (after rotation) and values as a bfloat16 KV cache holds
+                          * them (a property of the workload's storage, see layer_forward); 0: unrounded */
     double rms_eps, rope_theta;
     const void *embed;        /* [V][d] */
     const void *final_norm;   /* [d] */
@@ -672,7 +674,7 @@ void ora_tree_pass(const ora_model *m, const int32_t *tokens, const uint64_t *ma
             x[(size_t)t * d + i] = wget(m->embed, (size_t)tokens[t] * d + i, dt);
     for (int l = 0; l < m->n_layers; ++l)
         layer_forward(m, l, x, mask, pos, T, L, L_max, kc + (size_t)l * Hkv * L_max * D, vc + (size_t)l * Hkv * L_max * D,
-                      tree_k + (size_t)l * T * hkd, tree_v + (size_t)l * T * hkd, 0, &s);
+                      tree_k + (size_t)l * T * hkd, tree_v + (size_t)l * T * hkd, m->kv_bf16, &s);
     for (int t = 0; t < T; ++t)
         rmsnorm(x + (size_t)t * d, m->final_norm, dt, d, m->rms_eps, hidden + (size_t)t * d);
     if (logits)

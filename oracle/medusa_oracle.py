@@ -34,7 +34,7 @@ class _Model(C.Structure):
     _fields_ = [
         ("n_layers", C.c_int32), ("d", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
         ("ffn", C.c_int32), ("vocab", C.c_int32), ("n_medusa", C.c_int32), ("wdtype", C.c_int32),
-        ("n_kv_heads", C.c_int32), ("pad_", C.c_int32),
+        ("n_kv_heads", C.c_int32), ("kv_bf16", C.c_int32),
         ("rms_eps", C.c_double), ("rope_theta", C.c_double),
         ("embed", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p),
         ("layers", C.POINTER(C.c_void_p)),
@@ -205,7 +205,9 @@ LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up",
 class Model:
     """Holds numpy weights (float32, or uint16 bf16 bit patterns) and the C struct pointing at them."""
 
-    def __init__(self, cfg: dict, weights: dict):
+    def __init__(self, cfg: dict, weights: dict, kv_bf16: bool = False):
+        """kv_bf16: every pass holds its tree keys/values (and therefore everything committed to the cache) as a
+        bfloat16 KV cache holds them -- the storage precision the bf16 workloads define."""
         self.cfg = dict(cfg)
         self.w = weights
         any_w = np.ascontiguousarray(weights["lm_head"])
@@ -228,7 +230,8 @@ class Model:
         self._keep = keep
         self.c = _Model(
             n_layers=n_layers, d=cfg["d"], n_heads=cfg["n_heads"], head_dim=cfg["head_dim"], ffn=cfg["ffn"],
-            vocab=cfg["vocab"], n_medusa=cfg["n_medusa"], wdtype=wd, n_kv_heads=cfg.get("n_kv_heads", 0), pad_=0,
+            vocab=cfg["vocab"], n_medusa=cfg["n_medusa"], wdtype=wd, n_kv_heads=cfg.get("n_kv_heads", 0),
+            kv_bf16=1 if kv_bf16 else 0,
             rms_eps=cfg.get("rms_eps", 1e-5), rope_theta=cfg.get("rope_theta", 1e4),
             embed=ptr(weights["embed"]), final_norm=ptr(weights["final_norm"]), lm_head=ptr(weights["lm_head"]),
             layers=C.cast(arr, C.POINTER(C.c_void_p)),
