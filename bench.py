@@ -263,6 +263,8 @@ def run_gpu(args):
     torch.cuda.set_stream(stream)
     ctx = B.Context(cfg, B.BF16, WORKLOAD["L_max"], device=local, stream=stream.cuda_stream)
     tree = ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
+    if args.weight_prefetch is not None:
+        ctx.set_option(B.OPT_WEIGHT_PREFETCH, args.weight_prefetch)
     ctx.load_weights(dw)
     prompt = I.make_prompt(WORKLOAD["prompt"], cfg["vocab"], WORKLOAD["prompt_seed"])
     ctx.prefill(torch.from_numpy(prompt).cuda())
@@ -405,6 +407,7 @@ def run_gpu(args):
             "data": "synthetic",
             "config": {"workload": WORKLOAD["name"], "tree_nodes": T, "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"],
                        "cache_len_start": L0, "heads": cfg["n_medusa"], "replicas": world,
+                       "weight_prefetch_tiles": "library default" if args.weight_prefetch is None else args.weight_prefetch,
                        "l2": "inputs larger than L2: every step streams %.1f GB of weights" % (sb["gemm_weights"] / 1e9)},
             "clocks": clocks,
             "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": "tokens/s",
@@ -464,6 +467,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS), help="7b: the headline configuration")
+    ap.add_argument("--weight-prefetch", type=int, default=None, metavar="TILES",
+                    help="comparison runs: weight tiles per projection CTA that the in-between kernels pull into the L2 "
+                         "(library default if not given, 0 = off)")
     args = ap.parse_args()
     global WORKLOAD
     WORKLOAD = WORKLOADS[args.workload]

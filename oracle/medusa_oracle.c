@@ -34,7 +34,16 @@
 #include <stdlib.h>
 #include <string.h>
 
-#define ORA_MAX_T 64
+#define ORA_MAX_T 256
+
+/* Ancestor masks: node i owns W = ceil(T / 64) consecutive 64-bit words, bit j of the row (word j / 64, bit j % 64)
+ * says whether node j is visible to node i.  Trees of up to 64 nodes have one word per node. */
+static inline int mask_words(int T) { return (T + 63) / 64; }
+static inline int mask_bit(const uint64_t *mask, int W, int i, int j)
+{
+    return (int)((mask[(size_t)i * W + (j >> 6)] >> (j & 63)) & 1ull);
+}
+static inline void mask_set(uint64_t *mask, int W, int i, int j) { mask[(size_t)i * W + (j >> 6)] |= 1ull << (j & 63); }
 #define ORA_MAX_DEPTH 8
 
 /* ------------------------------------------------------------------ helpers */
@@ -270,7 +279,7 @@ int32_t ora_tree_paths_from_accuracies(const double *acc, int32_t depth, int32_t
  * Static tree buffers (Sec. 2.1.2, Fig. 2).  paths: [n_paths][max_depth] rank tuples, -1 padded,
  * distinct and prefix-closed.  Node 0 is the root (the LM head's own token); the other nodes are
  * sorted by (depth, tuple).  For node i:
- *   mask[i]     bit j set iff node j is i itself or one of its ancestors (root included)
+ *   mask[i]     bit j set iff node j is i itself or one of its ancestors (root included); ceil(T/64) words per node
  *   pos[i]      depth of i  (its rotary position is cache_len + pos[i])
  *   parent[i]   node index of the parent (-1 for the root)
  *   tree_idx[i] index into the candidate pool [root, head-1 ranks 0..topk-1, head-2 ranks ...]
@@ -311,7 +320,9 @@ int32_t ora_build_tree_buffers(const int32_t *paths, int32_t n_paths, int32_t ma
         order[b + 1] = cur;
     }
     int depth = 0, topk = 0;
-    mask[0] = 1ull;
+    const int W = mask_words(T);
+    memset(mask, 0, (size_t)T * W * sizeof(uint64_t));
+    mask_set(mask, W, 0, 0);
     pos[0] = 0;
     parent[0] = -1;
     tree_idx[0] = 0;
@@ -333,20 +344,20 @@ int32_t ora_build_tree_buffers(const int32_t *paths, int32_t n_paths, int32_t ma
     for (int i = 1; i < T; ++i) {
         const int32_t *ti = paths + (size_t)order[i - 1] * max_depth;
         int li = lens[order[i - 1]];
-        uint64_t m = 1ull | (1ull << i);
+        mask_set(mask, W, i, 0);
+        mask_set(mask, W, i, i);
         int par = li == 1 ? 0 : -1;
         for (int j = 1; j < i; ++j) {
             const int32_t *tj = paths + (size_t)order[j - 1] * max_depth;
             int lj = lens[order[j - 1]];
             if (lj < li && tuple_cmp(tj, lj, ti, lj) == 0) { /* tj is a proper prefix of ti */
-                m |= 1ull << j;
+                mask_set(mask, W, i, j);
                 if (lj == li - 1)
                     par = j;
             }
         }
         if (par < 0)
             return -4; /* not prefix-closed */
-        mask[i] = m;
         parent[i] = par;
         tree_idx[i] = 1 + (li - 1) * topk + ti[li - 1];
     }
@@ -453,7 +464,7 @@ void ora_expand_candidates(int32_t root, const int32_t *topk_idx /* [K][topk] */
  *   q, k_new, v_new : [T][H][D]  (already rotated)
  *   kc, vc          : [H][L_max][D], positions 0..L-1 valid (keys stored rotated)
  * Query i of head h sees every cache position 0..L-1 and then, in index order, the tree nodes
- * j with bit j of mask[i] set (its ancestors and itself).  out[i][h] = softmax(q.k/sqrt(D)) V.
+ * j with bit j of mask row i set (its ancestors and itself; ceil(T/64) words per row).  out[i][h] = softmax(q.k/sqrt(D)) V.
  * lse (nullable): [T][H] log-sum-exp of the scaled scores.
  */
 static void tree_attention_core(const double *q, const double *k_new, const double *v_new, const double *kc,
@@ -462,6 +473,7 @@ static void tree_attention_core(const double *q, const double *k_new, const doub
 {
     /* grouped-query attention: query head h reads key/value head h / (H / Hkv); Hkv == H is the ordinary case */
     const int group = H / Hkv;
+    const int W = mask_words(T);
     double scale = 1.0 / sqrt((double)D);
 #pragma omp parallel for collapse(2) schedule(static)
     for (int h = 0; h < H; ++h) {
@@ -472,7 +484,7 @@ static void tree_attention_core(const double *q, const double *k_new, const doub
             const int hk = h / group;
             double m = -INFINITY;
             for (int j = 0; j < nk; ++j) {
-                int visible = j < L || ((mask[i] >> (j - L)) & 1ull);
+                int visible = j < L || mask_bit(mask, W, i, j - L);
                 if (!visible) {
                     s[j] = -INFINITY;
                     continue;

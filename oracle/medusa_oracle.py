@@ -105,14 +105,16 @@ def tree_paths_from_accuracies(acc, n_nodes):
 
 
 def build_tree_buffers(paths, max_depth=None):
-    """-> dict(T, P, depth, topk, mask u64[T], pos, tree_idx, parent i32[T], retrieve i32[P][depth+1])"""
+    """-> dict(T, P, depth, topk, mask u64[T] (u64[T][ceil(T/64)] for trees of more than 64 nodes), pos, tree_idx,
+    parent i32[T], retrieve i32[P][depth+1])"""
     paths = _i32(paths)
     if paths.ndim == 1:
         paths = paths.reshape(0, max_depth or 1)
     n_paths, md = paths.shape
     T = n_paths + 1
     dims = np.zeros(4, dtype=np.int32)
-    mask = np.zeros(T, dtype=np.uint64)
+    W = (T + 63) // 64
+    mask = np.zeros(T * W, dtype=np.uint64)
     pos = np.zeros(T, dtype=np.int32)
     tree_idx = np.zeros(T, dtype=np.int32)
     parent = np.zeros(T, dtype=np.int32)
@@ -123,6 +125,8 @@ def build_tree_buffers(paths, max_depth=None):
         raise ValueError("ora_build_tree_buffers: invalid tree (code %d)" % rc)
     T, P, depth, topk = (int(x) for x in dims)
     retrieve = retrieve.reshape(-1)[: P * (depth + 1)].reshape(P, depth + 1).copy()
+    if W > 1:
+        mask = mask.reshape(T, W)
     return dict(T=T, P=P, depth=depth, topk=topk, mask=mask, pos=pos, tree_idx=tree_idx, parent=parent,
                 retrieve=retrieve)
 

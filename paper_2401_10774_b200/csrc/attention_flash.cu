@@ -19,6 +19,7 @@
 #include "common.cuh"
 #include "pdl.cuh"
 #include "kernels.h"
+#include "prefetch.cuh"
 
 namespace medusa {
 
@@ -27,11 +28,24 @@ namespace {
 constexpr int D = 128;          // head dim
 constexpr int BQ = 64;          // query rows per CTA (4 warps x 16)
 constexpr int BKEY = 64;        // keys per tile
-constexpr int STAGES = 3;
+#ifndef ATT_STAGES
+#define ATT_STAGES 3
+#endif
+#ifndef ATT_PREFETCH
+#define ATT_PREFETCH 1
+#endif
+#ifndef ATT_RANGES
+#define ATT_RANGES 1
+#endif
+#ifndef ATT_QLO
+#define ATT_QLO 1
+#endif
+constexpr int STAGES = ATT_STAGES;
 constexpr int THREADS = 256;     // 8 warps: warp w owns query rows 16*(w&3).. and key half (w>>2) of every tile
 constexpr int TILE_BYTES = BKEY * D * 2;           // 16 KiB for K, same for V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
-constexpr int SMEM_BYTES = TILE_BYTES + STAGES * STAGE_BYTES;   // Q tile, then the K/V ring
+constexpr int Q_BYTES = 2 * TILE_BYTES;                         // Q tile and its second plane (zeros without one)
+constexpr int SMEM_BYTES = Q_BYTES + STAGES * STAGE_BYTES;      // Q planes, then the K/V ring
 constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -71,6 +85,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 struct Args {
     const bf16 *q, *k_new, *v_new;   // [T][H][D]
+    const bf16 *q_lo;                // nullable [T][H][D]: second plane of q (scores are q.k + q_lo.k)
     const bf16 *k_cache, *v_cache;   // [H][L_max][D]
     const int32_t *cache_len;
     const uint64_t *mask;            // [T]
@@ -82,6 +97,7 @@ struct Args {
     int T, H, L_max, tiles_per_split, max_splits;
     int Hkv;                         // key/value heads; query head h reads key/value head h / (H / Hkv)
     int rows_max_tiles;              // caches of up to this many tiles run in row-split mode (0: never)
+    WeightPrefetch pf;               // weight tiles of the projection that follows, asked for before the dependency wait
 };
 
 // loads one 64-key tile pair (K and V) into a stage; rows >= n_valid are zero-filled
@@ -107,7 +123,8 @@ __device__ __forceinline__ void load_tile(uint8_t *stage, const bf16 *ksrc, cons
 // spelled out because one template for both measured 2-10 % slower (register allocation of the longer form).
 __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem_all, int h, int half, int L, int nt)
 {
-    uint8_t *smem = smem_all + TILE_BYTES;
+    uint8_t *smem = smem_all + Q_BYTES;
+    const bool has_qlo = a.q_lo != nullptr;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 1, kq = warp >> 1;
     const int rbase = half * 32;
@@ -133,6 +150,8 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
             const int r = idx >> 4, c = idx & 15;
             const bool ok = rbase + r < a.T;
             cp_async16(qb + tile_off(r, c), a.q + (size_t)(ok ? rbase + r : 0) * HD + (size_t)h * D + c * 8, ok);
+            if (has_qlo)
+                cp_async16(qb + TILE_BYTES + tile_off(r, c), a.q_lo + (size_t)(ok ? rbase + r : 0) * HD + (size_t)h * D + c * 8, ok);
         }
         cp_async_commit();
     }
@@ -144,12 +163,13 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
     cp_async_wait<STAGES - 1>();
     __syncthreads();
     uint32_t qf[8][4];
+    const int q_row = wq * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
+    const uint32_t q_lo_addr = smem_u32(smem_all) + TILE_BYTES;
     {
         const uint32_t qb = smem_u32(smem_all);
-        const int r = wq * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-            ldsm_x4(qb + tile_off(r, 2 * ks + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+            ldsm_x4(qb + tile_off(q_row, 2 * ks + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
     }
     const int lr0 = wq * 16 + g, lr1 = lr0 + 8;      // rows inside the half
     const int row0 = rbase + lr0, row1 = rbase + lr1;  // tree rows
@@ -180,6 +200,12 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
             ldsm_x4(kb + tile_off(kr, 2 * ks + ((lane >> 3) & 1)), b0, b1, b2, b3);
             mma_bf16(s[0], qf[ks], b0, b1);
             mma_bf16(s[1], qf[ks], b2, b3);
+            if (has_qlo) {  // the second plane's fragments come from shared memory: no registers to hold them
+                uint32_t ql[4];
+                ldsm_x4(q_lo_addr + tile_off(q_row, 2 * ks + (lane >> 4)), ql[0], ql[1], ql[2], ql[3]);
+                mma_bf16(s[0], ql, b0, b1);
+                mma_bf16(s[1], ql, b2, b3);
+            }
         }
         // ---- mask + online softmax (log2 domain)
         float mx0 = -INFINITY, mx1 = -INFINITY;
@@ -318,49 +344,110 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
     }
 }
 
+// The key ranges of a launch: which form runs, how many ranges, and one CTA's tiles -- all derived from the cache length.
+struct Ranges {
+    int L, nt, n_active, tile0, tile1, n_tiles;
+    bool rows_mode, has_tree, idle;
+};
+__device__ __forceinline__ Ranges plan_ranges(const Args &a, int L_raw, int sp)
+{
+    Ranges r;
+    // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
+    r.L = min(max(L_raw, 0), a.L_max);
+    r.nt = (r.L + BKEY - 1) / BKEY;
+    r.rows_mode = r.nt <= a.rows_max_tiles && gridDim.y >= 2;
+    // Key ranges: fixed by the launch (tiles_per_split > 0), or chosen here from the true cache length, so that the
+    // result does not depend on what the host knew about the length when it launched: as many ranges as the grid has
+    // rows (one wave of CTAs; every CTA requests its first tiles before the dependency wait, so a range costs little
+    // to start), but no range shorter than two tiles.
+    int tps = a.tiles_per_split;
+    if (tps <= 0) {
+#if ATT_RANGES == 1
+        const int want = min((int)gridDim.y, max(1, r.nt / 2));
+#else
+        int want = 1;
+        while (want * want < r.nt) ++want;
+        want = min(want, (int)gridDim.y);
+#endif
+        tps = r.nt > 0 ? (r.nt + want - 1) / want : 1;
+    }
+    const int n_cache_splits = (r.nt + tps - 1) / tps;
+    // never more ranges than the grid has rows: when the launch's fixed range size was chosen for a shorter cache than
+    // the one found here, the last range takes all the remaining tiles (slower, still complete)
+    r.n_active = min(n_cache_splits > 0 ? n_cache_splits : 1, (int)gridDim.y);
+    r.idle = sp >= r.n_active;
+    r.tile0 = sp * tps;
+    r.has_tree = sp == r.n_active - 1;
+    r.tile1 = r.has_tree ? r.nt : min(r.nt, r.tile0 + tps);
+    r.n_tiles = (r.tile1 - r.tile0) + (r.has_tree ? 1 : 0);
+    return r;
+}
+
 __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a)
 {
-    pdl_enter();
+    pdl_trigger();
     extern __shared__ __align__(1024) uint8_t smem_all[];
-    uint8_t *smem = smem_all + TILE_BYTES;  // K/V ring; the Q tile sits in front of it
+    uint8_t *smem = smem_all + Q_BYTES;  // K/V ring; the Q planes sit in front of it
+    const bool has_qlo = a.q_lo != nullptr;
     __shared__ int s_ticket;
     const int h = blockIdx.x, sp = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 3, kh = warp >> 2;  // query-row group, key half
-    // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
-    const int L = min(max(*a.cache_len, 0), a.L_max);
-    const int nt = (L + BKEY - 1) / BKEY;
-    if (nt <= a.rows_max_tiles && gridDim.y >= 2) {
+    const size_t HD = (size_t)a.H * D, HkvD = (size_t)a.Hkv * D;
+    const int hk = h / (a.H / a.Hkv);
+    // ---- before the dependency wait: request this CTA's first cache tiles.  The cache rows below the cache length, and
+    // the length itself, were written by the previous step's commit (or the prefill): kernels that had finished before
+    // the kernel in front of this one could start.  What the kernel in front writes are q and the tree's own keys and
+    // values, which are requested after the wait.  The length is read again after the wait; should it differ (never
+    // observed), the prefetched tiles are dropped and requested again.
+    Ranges rg = plan_ranges(a, *a.cache_len, sp);
+    bool waited = false;
+    auto prefetch_cache_tiles = [&]() {
+        if (rg.rows_mode || rg.idle)
+            return;
+#if !ATT_PREFETCH
+        if (!waited)
+            return;
+#endif
+        for (int i = 0; i < STAGES - 1; ++i) {
+            const int ct = rg.tile0 + i;
+            if (ct < rg.tile1) {
+                const size_t base = ((size_t)hk * a.L_max + (size_t)ct * BKEY) * D;
+                load_tile(smem + i * STAGE_BYTES, a.k_cache + base, a.v_cache + base, D, min(BKEY, rg.L - ct * BKEY));
+            }
+            cp_async_commit();
+        }
+    };
+    prefetch_cache_tiles();
+    prefetch_weights(a.pf, ((long long)blockIdx.y * gridDim.x + blockIdx.x) * THREADS + threadIdx.x,
+                     (long long)gridDim.x * gridDim.y * THREADS);
+    pdl_wait();
+    waited = true;
+#if !ATT_PREFETCH
+    rg = plan_ranges(a, *a.cache_len, sp);
+    prefetch_cache_tiles();
+#endif
+    {
+        const int L_now = min(max(*a.cache_len, 0), a.L_max);
+        if (L_now != rg.L) {
+            cp_async_wait<0>();
+            __syncthreads();
+            rg = plan_ranges(a, L_now, sp);
+            prefetch_cache_tiles();
+        }
+    }
+    const int L = rg.L, nt = rg.nt;
+    if (rg.rows_mode) {
         if (sp < 2)
             attention_rows_mode(a, smem_all, h, sp, L, nt);
         return;
     }
-    // Key ranges: fixed by the launch (tiles_per_split > 0), or chosen here from the true cache length, so that
-    // the result does not depend on what the host knew about the length when it launched.  A CTA's time grows
-    // with its tiles, the combine with the number of ranges: about sqrt(tiles) ranges balances the two, and never
-    // more ranges than the grid has rows.
-    int tps = a.tiles_per_split;
-    if (tps <= 0) {
-        int want = 1;
-        while (want * want < nt) ++want;
-        if (want > (int)gridDim.y) want = (int)gridDim.y;
-        tps = nt > 0 ? (nt + want - 1) / want : 1;
-    }
-    const int n_cache_splits = (nt + tps - 1) / tps;
-    // never more ranges than the grid has rows: when the launch's fixed range size was chosen for a shorter cache than
-    // the one found here, the last range takes all the remaining tiles (slower, still complete)
-    const int n_active = min(n_cache_splits > 0 ? n_cache_splits : 1, (int)gridDim.y);
-    if (sp >= n_active)
+    if (rg.idle)
         return;
-    const int tile0 = sp * tps;
-    const bool has_tree = sp == n_active - 1;
-    const int tile1 = has_tree ? nt : min(nt, tile0 + tps);
-    const int n_tiles = (tile1 - tile0) + (has_tree ? 1 : 0);
-    const size_t HD = (size_t)a.H * D, HkvD = (size_t)a.Hkv * D;
-    const int hk = h / (a.H / a.Hkv);
+    const int n_active = rg.n_active, tile0 = rg.tile0, tile1 = rg.tile1, n_tiles = rg.n_tiles;
 
     auto issue = [&](int i) {
-        // tile i of this CTA: a cache tile, or (last, if has_tree) the tree's own keys
+        // tile i of this CTA: a cache tile, or (last, if this is the last range) the tree's own keys
         uint8_t *stage = smem + (i % STAGES) * STAGE_BYTES;
         const int ct = tile0 + i;
         if (ct < tile1) {
@@ -370,7 +457,7 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             load_tile(stage, a.k_new + (size_t)hk * D, a.v_new + (size_t)hk * D, HkvD, a.T);
         }
     };
-    // ---- Q and the first K/V tiles are requested together; Q is copy group 0
+    // ---- after the wait: Q, and the tree's own tile if it is one of the first STAGES-1 tiles, as one more copy group
     {
         const uint32_t qb = smem_u32(smem_all);
 #pragma unroll
@@ -379,23 +466,23 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             int r = idx >> 4, c = idx & 15;
             bool ok = r < a.T;
             cp_async16(qb + tile_off(r, c), a.q + (size_t)(ok ? r : 0) * HD + (size_t)h * D + c * 8, ok);
+            if (has_qlo)
+                cp_async16(qb + TILE_BYTES + tile_off(r, c), a.q_lo + (size_t)(ok ? r : 0) * HD + (size_t)h * D + c * 8, ok);
         }
+        if (rg.has_tree && n_tiles - 1 < STAGES - 1)
+            issue(n_tiles - 1);
         cp_async_commit();
     }
-    for (int i = 0; i < STAGES - 1; ++i) {
-        if (i < n_tiles)
-            issue(i);
-        cp_async_commit();
-    }
-    cp_async_wait<STAGES - 1>();  // everything but the K/V groups just issued: Q has landed
+    cp_async_wait<0>();  // Q and the first STAGES-1 tiles have landed
     __syncthreads();
     uint32_t qf[8][4];
+    const int q_row = wq * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
+    const uint32_t q_lo_addr = smem_u32(smem_all) + TILE_BYTES;
     {
         const uint32_t qb = smem_u32(smem_all);
-        const int r = wq * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-            ldsm_x4(qb + tile_off(r, 2 * ks + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+            ldsm_x4(qb + tile_off(q_row, 2 * ks + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
     }
 
     const int row0 = wq * 16 + g, row1 = row0 + 8;
@@ -424,6 +511,9 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
+            uint32_t ql[4];
+            if (has_qlo)  // the second plane's fragments come from shared memory: no registers to hold them
+                ldsm_x4(q_lo_addr + tile_off(q_row, 2 * ks + (lane >> 4)), ql[0], ql[1], ql[2], ql[3]);
 #pragma unroll
             for (int np = 0; np < 2; ++np) {
                 uint32_t b0, b1, b2, b3;
@@ -431,6 +521,10 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
                 ldsm_x4(kb + tile_off(kr, 2 * ks + ((lane >> 3) & 1)), b0, b1, b2, b3);
                 mma_bf16(s[2 * np], qf[ks], b0, b1);
                 mma_bf16(s[2 * np + 1], qf[ks], b2, b3);
+                if (has_qlo) {
+                    mma_bf16(s[2 * np], ql, b0, b1);
+                    mma_bf16(s[2 * np + 1], ql, b2, b3);
+                }
             }
         }
         // ---- mask + online softmax (log2 domain)
@@ -595,78 +689,72 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     __syncthreads();
     if (s_ticket != n_active - 1)
         return;
-    // ---- last CTA of this head: combine the key ranges in split order
+    // ---- last CTA of this head: combine the key ranges in range order.  Thread -> 4 adjacent columns of 8 rows.  Every
+    // thread reads its rows' (max, sum) records itself (the lanes of a warp read the same 64 bytes: one broadcast
+    // transaction) together with the partial outputs, two ranges per round, all loads of a round in flight at once, and
+    // folds them in with a running maximum: one trip to the L2 instead of a staged max / weight / output sequence.
     __threadfence();
-    float (*s_w)[BQ] = reinterpret_cast<float (*)[BQ]>(smem);  // [max_splits + 1][64] weights; the ring is idle now
-    float *s_ml = reinterpret_cast<float *>(smem) + (FLASH_MAX_SPLITS + 1) * BQ;  // staged (max, sum) pairs [split][2][64]
     const float *__restrict__ mlh = a.ws_ml + (size_t)h * a.max_splits * 2 * BQ;
-    {
-        // one batch of independent loads: thread t fetches element t of every key range's 128-float record
-        float t[FLASH_MAX_SPLITS];
-        const bool mine = threadIdx.x < 2 * BQ;
-#pragma unroll
-        for (int s2 = 0; s2 < FLASH_MAX_SPLITS; ++s2)
-            if (mine && s2 < n_active) t[s2] = mlh[(size_t)s2 * 2 * BQ + threadIdx.x];
-#pragma unroll
-        for (int s2 = 0; s2 < FLASH_MAX_SPLITS; ++s2)
-            if (mine && s2 < n_active) s_ml[s2 * 2 * BQ + threadIdx.x] = t[s2];
-    }
-    __syncthreads();
-    if (threadIdx.x < BQ) {
-        const int r = threadIdx.x;
-        float mstar = -INFINITY;
-        for (int s2 = 0; s2 < n_active; ++s2)
-            mstar = fmaxf(mstar, s_ml[s2 * 2 * BQ + r]);
-        const float msafe = mstar == -INFINITY ? 0.f : mstar;
-        float lstar = 0.f;
-        for (int s2 = 0; s2 < n_active; ++s2) {
-            const float w = exp2f(s_ml[s2 * 2 * BQ + r] - msafe);
-            s_w[s2][r] = w;
-            lstar += w * s_ml[s2 * 2 * BQ + BQ + r];
-        }
-        s_w[FLASH_MAX_SPLITS][r] = lstar > 0.f ? 1.0f / lstar : 0.f;
-        if (a.lse && r < a.T)
-            a.lse[(size_t)r * a.H + h] = mstar / LOG2E + logf(lstar);
-    }
-    __syncthreads();
-    // thread -> 4 adjacent columns of 8 rows; per key range the 8 row loads are in flight together
     const float *__restrict__ oh = a.ws_o + (size_t)h * a.max_splits * BQ * D;
-    const int c4 = (threadIdx.x & 31) * 4, rg = (threadIdx.x >> 5) * 8;
+    const int c4 = (threadIdx.x & 31) * 4, r8 = (threadIdx.x >> 5) * 8;
+    float mrun[8], lrun[8];
     float4 acc[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < 8; ++u) {
+        mrun[u] = -INFINITY;
+        lrun[u] = 0.f;
         acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     for (int s2 = 0; s2 < n_active; s2 += 2) {
-        // two key ranges (16 independent 16-byte loads per thread) in flight per round; always added in range order
-        float4 v[8], v2[8];
         const bool two = s2 + 1 < n_active;
+        float4 v[8], v2[8], pm[2], pl[2], qm[2], ql[2];
+        const float *rec = mlh + (size_t)s2 * 2 * BQ;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            pm[u] = *reinterpret_cast<const float4 *>(rec + r8 + 4 * u);
+            pl[u] = *reinterpret_cast<const float4 *>(rec + BQ + r8 + 4 * u);
+        }
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            v[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)s2 * BQ + rg + u) * D + c4);
+            v[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)s2 * BQ + r8 + u) * D + c4);
         if (two) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                qm[u] = *reinterpret_cast<const float4 *>(rec + 2 * BQ + r8 + 4 * u);
+                ql[u] = *reinterpret_cast<const float4 *>(rec + 3 * BQ + r8 + 4 * u);
+            }
 #pragma unroll
             for (int u = 0; u < 8; ++u)
-                v2[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)(s2 + 1) * BQ + rg + u) * D + c4);
+                v2[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)(s2 + 1) * BQ + r8 + u) * D + c4);
         }
+        const float *pmf = reinterpret_cast<const float *>(pm), *plf = reinterpret_cast<const float *>(pl);
+        const float *qmf = reinterpret_cast<const float *>(qm), *qlf = reinterpret_cast<const float *>(ql);
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const float w = s_w[s2][rg + u];
-            acc[u].x += w * v[u].x; acc[u].y += w * v[u].y; acc[u].z += w * v[u].z; acc[u].w += w * v[u].w;
-        }
-        if (two) {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const float w = s_w[s2 + 1][rg + u];
-                acc[u].x += w * v2[u].x; acc[u].y += w * v2[u].y; acc[u].z += w * v2[u].z; acc[u].w += w * v2[u].w;
+            const float ma = pmf[u], mb = two ? qmf[u] : -INFINITY;
+            const float mn = fmaxf(mrun[u], fmaxf(ma, mb));
+            const float ms = mn == -INFINITY ? 0.f : mn;
+            const float c = exp2f(mrun[u] - ms), wa = exp2f(ma - ms), wb = exp2f(mb - ms);  // exp2f(-inf) = 0
+            mrun[u] = mn;
+            lrun[u] = lrun[u] * c + wa * plf[u] + (two ? wb * qlf[u] : 0.f);
+            acc[u].x = acc[u].x * c + wa * v[u].x;
+            acc[u].y = acc[u].y * c + wa * v[u].y;
+            acc[u].z = acc[u].z * c + wa * v[u].z;
+            acc[u].w = acc[u].w * c + wa * v[u].w;
+            if (two) {
+                acc[u].x += wb * v2[u].x;
+                acc[u].y += wb * v2[u].y;
+                acc[u].z += wb * v2[u].z;
+                acc[u].w += wb * v2[u].w;
             }
         }
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-        const int r = rg + u;
+        const int r = r8 + u;
         if (r >= a.T)
             continue;
-        const float inv = s_w[FLASH_MAX_SPLITS][r];
+        const float inv = lrun[u] > 0.f ? 1.0f / lrun[u] : 0.f;
         const float y[4] = {acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv};
         const size_t idx = (size_t)r * HD + (size_t)h * D + c4;
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]), h1 = __floats2bfloat162_rn(y[2], y[3]);
@@ -681,6 +769,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             pk.y = *reinterpret_cast<const uint32_t *>(&q1);
             *reinterpret_cast<uint2 *>(a.out_lo + idx) = pk;
         }
+        if (a.lse && c4 == 0)
+            a.lse[(size_t)r * a.H + h] = mrun[u] / LOG2E + logf(lrun[u]);
     }
     if (threadIdx.x == 0)
         a.counters[h] = 0;  // ready for the next launch
@@ -705,7 +795,7 @@ size_t tree_attention_flash_workspace_bytes(int H)
 cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                        int L_hint, cudaStream_t s)
+                                        int L_hint, cudaStream_t s, const void *q_lo, const WeightPrefetch *prefetch)
 {
     if (first_use_on_current_device(g_flash_attr_set)) {
         cudaError_t e = cudaFuncSetAttribute(tree_attention_flash_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -728,6 +818,7 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
     }
     Args a;
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
+    a.q_lo = ATT_QLO ? (const bf16 *)q_lo : nullptr;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
     a.cache_len = cache_len; a.mask = mask; a.out = (bf16 *)out; a.out_lo = (bf16 *)out_lo; a.lse = lse;
     a.ws_o = (float *)workspace;
@@ -735,6 +826,7 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
     a.counters = (int *)(a.ws_ml + (size_t)H * FLASH_MAX_SPLITS * 2 * BQ);
     a.T = T; a.H = H; a.Hkv = Hkv; a.L_max = L_max; a.tiles_per_split = tps; a.max_splits = FLASH_MAX_SPLITS;
     a.rows_max_tiles = rows_mode_max_tiles();
+    a.pf = prefetch ? *prefetch : WeightPrefetch{};
     dim3 grid(H, splits);
     launch_pdl(tree_attention_flash_kernel, dim3(grid), dim3(THREADS), SMEM_BYTES, s, a);
     return cudaGetLastError();
@@ -811,6 +903,7 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
     float *base = (float *)g_static_scratch_addr[dev];
     Args a;
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
+    a.q_lo = nullptr;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
     a.cache_len = cache_len; a.mask = mask; a.out = (bf16 *)out; a.out_lo = nullptr; a.lse = lse;
     a.ws_o = base;
@@ -830,6 +923,7 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
     }
     a.T = T; a.H = H; a.Hkv = H; a.L_max = L_max; a.tiles_per_split = tps; a.max_splits = STATIC_MAX_SPLITS;
     a.rows_max_tiles = rows_mode_max_tiles();
+    a.pf = WeightPrefetch{};
     cudaError_t e = launch_pdl(tree_attention_flash_kernel, dim3(H, splits), dim3(THREADS), (size_t)SMEM_BYTES, s, a);
     return e == cudaSuccess ? MEDUSA_OK : MEDUSA_ERR_CUDA;
 }

@@ -498,6 +498,29 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
     return pd;
 }
 
+WeightPrefetch gemm_tc_prefetch_plan(const void *const *W, int n_seg, int seg_cols, int K, bool whole_tiles, int seg0_cols,
+                                     int units)
+{
+    WeightPrefetch p{};
+    if (seg0_cols <= 0) seg0_cols = seg_cols;
+    if (K % BK != 0 || units <= 0 || !W)
+        return p;  // units = 0
+    const PlaneDesc pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, 0, seg0_cols);
+    for (int i = 0; i < 3; ++i) p.W[i] = W[i < n_seg ? i : 0];
+    p.n_seg = n_seg;
+    p.seg0_tiles = (seg0_cols + BM - 1) / BM;
+    p.seg_tiles = (seg_cols + BM - 1) / BM;
+    p.seg0_rows = seg0_cols;
+    p.seg_rows = seg_cols;
+    p.K = K;
+    p.KB = pd.KB;
+    p.G = pd.ctas;
+    p.whole_tiles = whole_tiles ? 1 : 0;
+    p.total = pd.total;
+    p.units = units;
+    return p;
+}
+
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
                            int seg0_cols, uint32_t spin_limit, int withhold)

@@ -55,6 +55,19 @@ struct GemmTcArgs {
     int withhold;            // test hook: CTA 0's producer issues no load at all, so its consumers' waits expire
 };
 
+// What a kernel that runs before a projection launch needs to know to pull that launch's first weight tiles into the
+// L2 (prefetch.cuh).  units == 0: nothing to prefetch.
+struct WeightPrefetch {
+    const void *W[3];        // weight matrices of the launch ([rows][K] bf16)
+    int n_seg, seg0_tiles, seg_tiles, seg0_rows, seg_rows;
+    int K, KB, G, whole_tiles;
+    long long total;         // tiles * KB
+    int units;               // (tile, k block) pairs per CTA to prefetch
+};
+// plan of the prefetch for a launch described like gemm_tc_plan's; K must be a multiple of 64 (else units = 0)
+WeightPrefetch gemm_tc_prefetch_plan(const void *const *W, int n_seg, int seg_cols, int K, bool whole_tiles, int seg0_cols,
+                                     int units);
+
 // W: [N][K] bf16 row-major
 bool make_weight_map(TensorMap *out, const void *W, int N, int K);
 // X_planes: split activation, [2][64][K] bf16

@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "pdl.cuh"
 #include "kernels.h"
+#include "prefetch.cuh"
 
 namespace medusa {
 
@@ -124,9 +125,11 @@ template <typename WT, int GROUPS, int MAXT>
 __global__ void __launch_bounds__(MAXT)
 rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ planes, PlaneDesc pd,
                const WT *__restrict__ gain, float eps, WT *__restrict__ out, WT *__restrict__ out_lo,
-               float *__restrict__ out_f32, int d)
+               float *__restrict__ out_f32, int d, WeightPrefetch pf)
 {
-    pdl_enter();
+    pdl_trigger();
+    prefetch_weights(pf, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+    pdl_wait();
     __shared__ float red[32];
     const int t = blockIdx.x;
     float *xr = x + (size_t)t * d;
@@ -176,25 +179,27 @@ rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ planes, PlaneDes
 
 template <typename WT, int GROUPS, int MAXT>
 static void launch_rmsnorm_as(float *x, const float *planes, const PlaneDesc &pd, const void *gain, float eps, void *out,
-                              void *out_lo, float *out_f32, int T, int d, cudaStream_t s)
+                              void *out_lo, float *out_f32, int T, int d, cudaStream_t s, const WeightPrefetch &pf)
 {
     int threads = ((d / (4 * GROUPS) + 31) / 32) * 32;
     if (threads > MAXT) threads = MAXT;
     launch_pdl(rmsnorm_kernel<WT, GROUPS, MAXT>, dim3(T), dim3(threads), 0, s, x, planes, pd, (const WT *)gain, eps,
-               (WT *)out, (WT *)out_lo, out_f32, d);
+               (WT *)out, (WT *)out_lo, out_f32, d, pf);
 }
 
 void launch_add_rmsnorm(int dtype, float *x, const float *planes, const PlaneDesc &pd, const void *gain,
-                        float eps, void *out, void *out_lo, float *out_f32, int T, int d, cudaStream_t s)
+                        float eps, void *out, void *out_lo, float *out_f32, int T, int d, cudaStream_t s,
+                        const WeightPrefetch *prefetch)
 {
+    const WeightPrefetch pf = prefetch ? *prefetch : WeightPrefetch{};
     // rows of up to 4096 columns: one column group per thread; wider rows: two groups per thread in blocks of at
     // most 768 threads, which leaves the compiler 80 registers for both groups' loads in flight
     if (dtype == MEDUSA_BF16) {
-        if (d <= 4096) launch_rmsnorm_as<bf16, 1, 1024>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s);
-        else launch_rmsnorm_as<bf16, 2, 768>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s);
+        if (d <= 4096) launch_rmsnorm_as<bf16, 1, 1024>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s, pf);
+        else launch_rmsnorm_as<bf16, 2, 768>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s, pf);
     } else {
-        if (d <= 4096) launch_rmsnorm_as<float, 1, 1024>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s);
-        else launch_rmsnorm_as<float, 2, 768>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s);
+        if (d <= 4096) launch_rmsnorm_as<float, 1, 1024>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s, pf);
+        else launch_rmsnorm_as<float, 2, 768>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s, pf);
     }
 }
 
@@ -318,7 +323,7 @@ void launch_rope_table(float2 *cs, const int32_t *cache_len, const int32_t *pos,
 template <typename AT>
 __global__ void __launch_bounds__(256)
 rope_split_kernel(const float *__restrict__ qkv, PlaneDesc pd_q, PlaneDesc pd_kv, int kv_col0, const float2 *__restrict__ cs,
-                  AT *__restrict__ q, AT *__restrict__ tk, AT *__restrict__ tv, int H, int Hkv, int D)
+                  AT *__restrict__ q, AT *__restrict__ q_lo, AT *__restrict__ tk, AT *__restrict__ tv, int H, int Hkv, int D)
 {
     pdl_enter();
     const int t = blockIdx.y, which = blockIdx.z, half = D / 2, per_head = half / 4;
@@ -363,22 +368,25 @@ rope_split_kernel(const float *__restrict__ qkv, PlaneDesc pd_q, PlaneDesc pd_kv
     float y0[4], y1[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) { y0[i] = xa[i] * cc[i] - xb[i] * sn[i]; y1[i] = xb[i] * cc[i] + xa[i] * sn[i]; }
+    // q may be kept as two planes (hi + lo), so that the scores do not carry q's rounding to one plane; keys are a
+    // cache format (one plane by definition)
     AT *dst = which == 0 ? q : tk;
-    store_split4<AT>(dst, nullptr, o, y0);
-    store_split4<AT>(dst, nullptr, o + half, y1);
+    AT *dst_lo = which == 0 ? q_lo : nullptr;
+    store_split4<AT>(dst, dst_lo, o, y0);
+    store_split4<AT>(dst, dst_lo, o + half, y1);
 }
 
 void launch_rope_split(int dtype, const float *qkv, const PlaneDesc &pd_q, const PlaneDesc &pd_kv, int kv_col0, const float2 *cs,
-                       void *q, void *tree_k, void *tree_v, int T, int H, int Hkv, int D, cudaStream_t s)
+                       void *q, void *q_lo, void *tree_k, void *tree_v, int T, int H, int Hkv, int D, cudaStream_t s)
 {
     const int n = H * (D / 8);
     dim3 grid((n + 255) / 256, T, 3);
     if (dtype == MEDUSA_BF16)
-        launch_pdl(rope_split_kernel<bf16>, dim3(grid), dim3(256), 0, s, qkv, pd_q, pd_kv, kv_col0, cs, (bf16 *)q, (bf16 *)tree_k,
-                   (bf16 *)tree_v, H, Hkv, D);
+        launch_pdl(rope_split_kernel<bf16>, dim3(grid), dim3(256), 0, s, qkv, pd_q, pd_kv, kv_col0, cs, (bf16 *)q, (bf16 *)q_lo,
+                   (bf16 *)tree_k, (bf16 *)tree_v, H, Hkv, D);
     else
-        launch_pdl(rope_split_kernel<float>, dim3(grid), dim3(256), 0, s, qkv, pd_q, pd_kv, kv_col0, cs, (float *)q, (float *)tree_k,
-                   (float *)tree_v, H, Hkv, D);
+        launch_pdl(rope_split_kernel<float>, dim3(grid), dim3(256), 0, s, qkv, pd_q, pd_kv, kv_col0, cs, (float *)q, (float *)nullptr,
+                   (float *)tree_k, (float *)tree_v, H, Hkv, D);
 }
 
 template <typename AT>
@@ -410,9 +418,12 @@ void launch_rope_apply(int dtype, const void *in, const float2 *cs, void *out, i
 template <typename AT>
 __global__ void __launch_bounds__(256)
 silu_mul_kernel(const float *__restrict__ gu, PlaneDesc pd, AT *__restrict__ act, AT *__restrict__ act_lo,
-                int F)
+                int F, WeightPrefetch pf)
 {
-    pdl_enter();
+    pdl_trigger();
+    prefetch_weights(pf, ((long long)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x,
+                     (long long)gridDim.x * gridDim.y * blockDim.x);
+    pdl_wait();
     const int t = blockIdx.y;
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= F)
@@ -438,13 +449,14 @@ silu_mul_kernel(const float *__restrict__ gu, PlaneDesc pd, AT *__restrict__ act
 }
 
 void launch_silu_mul(int dtype, const float *gate_up, const PlaneDesc &pd, void *act, void *act_lo, int T,
-                     int F, cudaStream_t s)
+                     int F, cudaStream_t s, const WeightPrefetch *prefetch)
 {
+    const WeightPrefetch pf = prefetch ? *prefetch : WeightPrefetch{};
     dim3 grid((F / 4 + 255) / 256, T);
     if (dtype == MEDUSA_BF16)
-        launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, s, gate_up, pd, (bf16 *)act, (bf16 *)act_lo, F);
+        launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, s, gate_up, pd, (bf16 *)act, (bf16 *)act_lo, F, pf);
     else
-        launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, s, gate_up, pd, (float *)act, nullptr, F);
+        launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, s, gate_up, pd, (float *)act, (float *)nullptr, F, pf);
 }
 
 // ---------------------------------------------------------------------------------------- small helpers

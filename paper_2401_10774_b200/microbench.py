@@ -35,6 +35,7 @@ def main():
     ap.add_argument("--typical", action="store_true", help="typical acceptance (0.7 / 0.09 / 0.3) instead of greedy")
     ap.add_argument("--attention", type=int, default=0, metavar="L", help="time tree_attention alone at cache length L")
     ap.add_argument("--caches", type=int, default=32)
+    ap.add_argument("--weight-prefetch", type=int, default=None, metavar="TILES")
     args = ap.parse_args()
     if args.attention:
         return attention_only(args)
@@ -51,6 +52,8 @@ def main():
     dw["layers"] = [{k: dev(v) for k, v in lw.items()} for lw in w["layers"]]
     ctx = B.Context(cfg, B.BF16, args.L_max)
     ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
+    if args.weight_prefetch is not None:
+        ctx.set_option(B.OPT_WEIGHT_PREFETCH, args.weight_prefetch)
     ctx.load_weights(dw)
     # a cache of the requested length without paying for a long prefill: prefill 64 tokens, then tell the
     # library the rest is there (the K/V values beyond are zeros, which is fine for timing)

@@ -52,7 +52,7 @@ class _OracleRun:
         c = o.accept_and_update_kv(p["tree_k"], p["tree_v"], self.kc, self.vc, r["acc_nodes"], r["accept_len"], 1 << 20,
                                    self.L, p["hidden"], tok)
         self.L, self.h_last, self.root = c["L"], c["h_last"], r["next_root"]
-        return [int(t) for t in c["emitted"]], lg, r
+        return [int(t) for t in c["emitted"]], lg, r, tok
 
 
 CONFIGS = [
@@ -156,15 +156,18 @@ def test_decode_configuration_stagewise_and_token_stream(oracle, case):
         assert em.tolist() == tok[acc[:n]].tolist()
         # ---- the oracle's own stream
         if run is not None and first_divergence is None and s < oracle_steps:
-            o_em, o_lg, o_r = run.step(o_mode, f32(tau), f32(eps), f32(delta), None if noise is None else noise[s])
+            o_em, o_lg, o_r, o_tok = run.step(o_mode, f32(tau), f32(eps), f32(delta), None if noise is None else noise[s])
             if o_em != em.tolist() or o_r["next_root"] != st["root"]:
                 # the deciding position: the first node whose decision differs; report the GPU's top-2 gap there
                 node = int(acc[min(len(o_em), n) - 1])
                 gap = _top2_gap(lg[node])
                 first_divergence = dict(step=s, gpu=em.tolist(), oracle=o_em, node=node, top2_gap=gap)
             else:
-                err = float(np.abs(lg - o_lg).max())
-                assert err <= TOL_LOGIT_BF16 * 4, "step %d: logits drifted %.3g from the oracle's own run" % (s, err)
+                # rows whose whole root-to-node token path is the same on both sides see the same context (the heads'
+                # near-ties may give the two sides different candidates elsewhere in the tree): the root always does
+                same = [i for i in range(T) if all(tok[j] == o_tok[j] for j in range(T) if (int(ot["mask"][i]) >> j) & 1)]
+                err = float(np.abs(lg[same] - o_lg[same]).max())
+                assert 0 in same and err <= TOL_LOGIT_BF16 * 4, "step %d: logits drifted %.3g from the oracle's own run" % (s, err)
         L += n
         lens.append(n)
     print("%s: %d steps, tokens per step mean %.2f max %d, min typical margin %.3g, first divergence from the oracle's own run: %s"

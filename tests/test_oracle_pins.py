@@ -654,3 +654,86 @@ def test_layer_entry_composes_to_the_tree_pass_and_bf16_storage_rounding(oracle)
     # the LM head alone on a given hidden state
     alone = oracle.final_norm_lm_head(om, hidden_in=ref["hidden"])
     assert np.array_equal(alone["logits"], ref["logits"])
+
+
+# ----------------------------------------------------------------------------- trees of more than 64 nodes (Sec. 3.3.1, Fig. 4)
+
+def _independent_top_n_tree(per_depth_topk, n_nodes):
+    """The surrogate sparse tree worked out a second way: enumerate the Cartesian tree, sort every node by (integer
+    denominator prod(i_j + 1) ascending, tuple ascending with a prefix before its extensions), keep the best n - 1.
+    Scores never increase along a path and a prefix sorts first, so the cut is prefix-closed and equals what greedy
+    node adding (Sec. 2.3.3) selects."""
+    nodes = []
+    for k in range(1, len(per_depth_topk) + 1):
+        nodes += list(itertools.product(*[range(s) for s in per_depth_topk[:k]]))
+    nodes.sort(key=lambda n: (math.prod(i + 1 for i in n), n))
+    return set(nodes[: n_nodes - 1])
+
+
+def _row_bits(mask_row):
+    """Set bits of a multi-word mask row (word w holds nodes 64 w .. 64 w + 63)."""
+    words = np.atleast_1d(mask_row)
+    return {64 * w + b for w, word in enumerate(words) for b in range(64) if (int(word) >> b) & 1}
+
+
+@pytest.mark.parametrize("topk,n_nodes", [((6, 4, 3, 2, 2), 128), ((10, 6, 4, 3, 2), 256), ((8, 8), 73)])
+def test_large_tree_buffers_against_an_independent_construction(oracle, topk, n_nodes):
+    paths = oracle.default_tree_paths(topk, n_nodes)
+    got = {tuple(int(x) for x in p if x >= 0) for p in paths}
+    assert got == _independent_top_n_tree(topk, n_nodes)
+    t = oracle.build_tree_buffers(paths)
+    T = t["T"]
+    assert T == n_nodes and t["mask"].shape == (T, (T + 63) // 64)
+    # node order: root first, then (depth, tuple); masks = the ancestor sets found by walking the parent pointers
+    order = [()] + sorted(got, key=lambda n: (len(n), n))
+    index = {n: i for i, n in enumerate(order)}
+    for i, n in enumerate(order):
+        anc = {index[n[:k]] for k in range(len(n) + 1)}
+        assert _row_bits(t["mask"][i]) == anc
+        assert t["pos"][i] == len(n)
+        assert t["parent"][i] == (index[n[:-1]] if n else -1)
+        assert t["tree_idx"][i] == (1 + (len(n) - 1) * t["topk"] + n[-1] if n else 0)
+    leaves = sorted(n for n in order if not any(m[:-1] == n for m in got if m))
+    assert t["P"] == len(leaves)
+    for r, leaf in enumerate(leaves):
+        want = [index[leaf[:k]] for k in range(len(leaf) + 1)]
+        assert [int(x) for x in t["retrieve"][r] if x >= 0] == want
+
+
+@pytest.mark.parametrize("topk,n_nodes,L", [((6, 4, 3, 2, 2), 128, 9), ((10, 6, 4, 3, 2), 256, 0), ((7, 5, 3), 100, 33)])
+def test_large_tree_attention_equals_per_path_causal_attention(oracle, topk, n_nodes, L):
+    # the invariant that defines tree attention, on trees whose masks span several 64-bit words: for every
+    # root-to-leaf path, ordinary causal attention over [cache; path] reproduces the outputs of the path's nodes
+    H, D, L_max = 2, 16, 40
+    t = oracle.build_tree_buffers(oracle.default_tree_paths(topk, n_nodes))
+    T = t["T"]
+    a = I.attention_inputs(T, H, D, L, L_max, 24, dtype="f32")
+    out, lse = oracle.tree_attention(a["q"], a["k_new"], a["v_new"], a["k_cache"], a["v_cache"], L, t["mask"],
+                                     t["pos"], apply_rope=True)
+    q = np.stack([[oracle.rope(a["q"][i, h], L + t["pos"][i]) for h in range(H)] for i in range(T)])
+    k = np.stack([[oracle.rope(a["k_new"][i, h], L + t["pos"][i]) for h in range(H)] for i in range(T)])
+    covered = set()
+    for row in t["retrieve"]:
+        row = [int(x) for x in row if x >= 0]
+        covered |= set(row)
+        for h in range(H):
+            kk = np.concatenate([a["k_cache"][h, :L].astype(np.float64), k[row, h]], axis=0)
+            vv = np.concatenate([a["v_cache"][h, :L].astype(np.float64), a["v_new"][row, h].astype(np.float64)])
+            qq = np.concatenate([np.zeros((L, D)), q[row, h]], axis=0)
+            ref = _sdpa(qq[None], kk[None], vv[None], causal=True)[0][L:]
+            np.testing.assert_allclose(out[row, h], ref, rtol=0, atol=1e-12)
+    assert covered == set(range(T)) and np.all(np.isfinite(lse))
+
+
+def test_large_tree_medusa_greedy_equals_plain_greedy(oracle):
+    # the exactness property of greedy acceptance does not depend on the tree's size: a 100-node tree on the tiny model
+    cfg = I.model_shape("tiny", n_medusa=3)
+    w = I.make_weights(cfg, seed=0, dtype="f32", head_init="lm_copy")
+    om = oracle.Model(cfg, w)
+    t = oracle.build_tree_buffers(oracle.default_tree_paths((7, 5, 3), 100))
+    prompt = I.make_prompt(20, cfg["vocab"], 1)
+    G = 24
+    ref = oracle.generate(om, t, prompt, G, 64, mode=oracle.GREEDY)
+    plain = oracle.generate_plain(om, prompt, G, 64)
+    assert ref["tokens"].tolist() == plain["tokens"].tolist()
+    assert ref["emitted_per_step"].sum() == G and ref["emitted_per_step"].max() <= t["depth"] + 1
