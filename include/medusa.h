@@ -54,13 +54,18 @@ typedef struct {
                          * query head h reads key/value head h / (n_heads / n_kv_heads), wk and wv have
                          * n_kv_heads*head_dim rows, and every K/V tensor below has n_kv_heads in place of H */
     float rms_eps, rope_theta;
+    int32_t max_tree_nodes; /* largest tree (nodes incl. root) the context must hold; 0 = 64.  Up to 256 (paper Sec. 3.3.1 /
+                             * Fig. 4 studies trees of that size): buffers are sized for ceil(max/64) tiles of 64 token
+                             * rows, projections and attention then run tile by tile */
 } medusa_model_desc;
 
 /* Static tree buffers (paper Sec. 2.1.2, Fig. 2).  Host arrays owned by the caller:
- * mask/pos/tree_idx/parent hold >= n_paths+1 entries, retrieve >= (n_paths+1)*(max_depth+1). */
+ * pos/tree_idx/parent hold >= n_paths+1 entries, mask >= (n_paths+1)*ceil((n_paths+1)/64), retrieve >=
+ * (n_paths+1)*(max_depth+1). */
 typedef struct {
     int32_t T, P, depth, topk; /* out: nodes incl. root, leaves, deepest level, max rank+1 */
-    uint64_t *mask;            /* [T]  bit j of mask[i]: node j is i or an ancestor of i */
+    uint64_t *mask;            /* [T][W], W = ceil(T/64) words per node: bit j of row i (word j/64, bit j%64) says node j is
+                                * i or an ancestor of i.  Trees of up to 64 nodes: one word per node */
     int32_t *pos;              /* [T]  depth of the node = rotary position offset from the cache length */
     int32_t *tree_idx;         /* [T]  index into the candidate pool [root, head1 top-k, head2 top-k, ...] */
     int32_t *parent;           /* [T]  parent node, -1 for the root */
@@ -90,8 +95,10 @@ typedef struct {
 enum {
     MEDUSA_WS_LOGITS = 0,   /* float [T][V]   backbone logits of the last tree pass */
     MEDUSA_WS_HIDDEN = 1,   /* float [T][d]   final-norm output of the last tree pass */
-    MEDUSA_WS_TREE_K = 2,   /* dtype [N_L][64][Hkv][D] rotated keys of the last tree pass (T rows used per layer) */
-    MEDUSA_WS_TREE_V = 3,   /* dtype [N_L][64][Hkv][D] */
+    MEDUSA_WS_TREE_K = 2,   /* dtype [N_L][R][Hkv][D] rotated keys of the last tree pass (T rows used per layer); R = the
+                             * context's token rows: 64, or 64*ceil(max_tree_nodes/64) -- also the row count of LOGITS,
+                             * HIDDEN and the TAP buffers */
+    MEDUSA_WS_TREE_V = 3,   /* dtype [N_L][R][Hkv][D] */
     MEDUSA_WS_K_CACHE = 4,  /* dtype [N_L][Hkv][L_max][D] */
     MEDUSA_WS_V_CACHE = 5,  /* dtype [N_L][Hkv][L_max][D] */
     MEDUSA_WS_HEAD_LOGITS = 6, /* float [K][V]  Medusa-head logits of the last step */
@@ -134,7 +141,7 @@ enum {
 /* Creates a context on CUDA device `device`; `stream` is a cudaStream_t.  With NULL the context creates a
  * blocking stream of its own (the legacy default stream cannot be captured into the whole-step graphs); like
  * every blocking stream it orders itself with work on the legacy default stream in both directions.
- * Shapes supported: head_dim in {64,128}, T <= 64, d and ffn multiples of 8 (bf16) / 4 (f32). */
+ * Shapes supported: head_dim in {64,128}, T <= max_tree_nodes <= 256, d and ffn multiples of 8 (bf16) / 4 (f32). */
 int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc, int32_t device, void *stream);
 int32_t medusa_destroy(medusa_ctx *ctx);
 const char *medusa_last_error(const medusa_ctx *ctx);
@@ -187,14 +194,14 @@ int32_t medusa_default_tree_paths(const int32_t *per_depth_topk_host, int32_t de
  * medusa_build_tree_buffers).  expected_len_host_out (nullable): the sum of the chosen nodes' accuracies, i.e.
  * the expected number of accepted speculated tokens per step under the independence assumption.
  * Host-only, allocates only host memory.  Returns the number of paths, or INVALID_ARG (null, sizes < 1, depth > 8,
- * an accuracy outside [0, 1] or NaN) / SHAPE (n_nodes > 64 or more nodes asked for than the Cartesian tree has). */
+ * an accuracy outside [0, 1] or NaN) / SHAPE (n_nodes > 256 or more nodes asked for than the Cartesian tree has). */
 int32_t medusa_tree_paths_from_accuracies(const double *acc_host, int32_t depth, int32_t topk, int32_t n_nodes,
                                           int32_t *paths_host_out, double *expected_len_host_out);
 
 /* paths_host: [n_paths][max_depth] rank tuples (0-based rank of head j's prediction at depth j), -1 padded,
- * distinct and prefix-closed; T = n_paths+1 <= 64.  Fills out_host (node 0 = root, others sorted by
+ * distinct and prefix-closed; T = n_paths+1 <= 256 (and <= the context's max_tree_nodes, 64 by default).  Fills out_host (node 0 = root, others sorted by
  * (depth, tuple)) and, if ctx != NULL, uploads a device copy that the other calls use.
- * Errors: INVALID_ARG (null), SHAPE (T > 64, depth > 8, depth > n_medusa), INVALID_ARG (not prefix-closed,
+ * Errors: INVALID_ARG (null), SHAPE (T > 256 or > the context's capacity, depth > 8, depth > n_medusa), INVALID_ARG (not prefix-closed,
  * duplicate, hole in padding). */
 int32_t medusa_build_tree_buffers(medusa_ctx *ctx, const int32_t *paths_host, int32_t n_paths, int32_t max_depth,
                                   medusa_tree_buffers *out_host);
@@ -266,7 +273,8 @@ int32_t medusa_evaluate_posterior(medusa_ctx *ctx, const float *logits, const in
 
 /* n = min(1 + *accept_len, max_commit).  For every layer: cache[:, L+j, :] <- tree[acc_nodes[j]], j < n;
  * emitted[j] = tree_tok[acc_nodes[j]]; *n_emitted = n; h_last <- hidden[acc_nodes[n-1]]; *cache_len += n.
- * tree_k, tree_v: [N_L][64][Hkv][D] (row stride fixed at 64 nodes); caches: [N_L][Hkv][L_max][D];
+ * tree_k, tree_v: [N_L][R][Hkv][D] (R = the context's token rows: 64 unless max_tree_nodes asks for more); caches:
+ * [N_L][Hkv][L_max][D];
  * hidden: float [T][d]; h_last: float [d].  If L + n > L_max nothing is written and the device status becomes
  * MEDUSA_ERR_CACHE_FULL. */
 int32_t medusa_accept_and_update_kv(medusa_ctx *ctx, const void *tree_k, const void *tree_v, void *k_cache,

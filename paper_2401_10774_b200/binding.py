@@ -33,7 +33,8 @@ class MedusaError(RuntimeError):
 class ModelDesc(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("ffn", C.c_int32), ("vocab", C.c_int32), ("n_medusa", C.c_int32), ("dtype", C.c_int32),
-                ("L_max", C.c_int32), ("n_kv_heads", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float)]
+                ("L_max", C.c_int32), ("n_kv_heads", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float),
+                ("max_tree_nodes", C.c_int32)]
 
 
 class TreeBuffers(C.Structure):
@@ -112,7 +113,8 @@ def build_tree_buffers(ctx, paths, max_depth=None) -> dict:
         paths = paths.reshape(0, max_depth or 1)
     n_paths, md = paths.shape
     T = n_paths + 1
-    mask = np.zeros(T, dtype=np.uint64)
+    W = (T + 63) // 64
+    mask = np.zeros(T * W, dtype=np.uint64)
     pos, tree_idx, parent = (np.zeros(T, dtype=np.int32) for _ in range(3))
     retrieve = np.full(T * (md + 1), -1, dtype=np.int32)
     tb = TreeBuffers(mask=mask.ctypes.data, pos=pos.ctypes.data, tree_idx=tree_idx.ctypes.data,
@@ -121,6 +123,8 @@ def build_tree_buffers(ctx, paths, max_depth=None) -> dict:
     rc = lib().medusa_build_tree_buffers(h, _ptr(paths), C.c_int32(n_paths), C.c_int32(md), C.byref(tb))
     if rc != OK:
         raise MedusaError(rc, ctx.last_error() if ctx is not None else "invalid tree")
+    if W > 1:
+        mask = mask.reshape(T, W)
     tree = dict(T=tb.T, P=tb.P, depth=tb.depth, topk=tb.topk, mask=mask, pos=pos, tree_idx=tree_idx, parent=parent,
                 retrieve=retrieve[: tb.P * (tb.depth + 1)].reshape(tb.P, tb.depth + 1).copy())
     if ctx is not None:
@@ -139,7 +143,8 @@ class Context:
         self._keep = []
         desc = ModelDesc(n_layers=cfg["n_layers"], d=cfg["d"], n_heads=cfg["n_heads"], head_dim=cfg["head_dim"],
                          ffn=cfg["ffn"], vocab=cfg["vocab"], n_medusa=cfg["n_medusa"], dtype=dtype, L_max=L_max,
-                         n_kv_heads=cfg.get("n_kv_heads", 0), rms_eps=cfg.get("rms_eps", 1e-5), rope_theta=cfg.get("rope_theta", 1e4))
+                         n_kv_heads=cfg.get("n_kv_heads", 0), rms_eps=cfg.get("rms_eps", 1e-5), rope_theta=cfg.get("rope_theta", 1e4),
+                         max_tree_nodes=cfg.get("max_tree_nodes", 0))
         self.handle = C.c_void_p(0)
         sp = C.c_void_p(0 if stream is None else int(stream))
         rc = lib().medusa_create(C.byref(self.handle), C.byref(desc), C.c_int32(device), sp)

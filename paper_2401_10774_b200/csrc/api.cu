@@ -21,6 +21,7 @@ using namespace medusa;
 struct medusa_ctx {
     medusa_model_desc m{};
     int device = 0;
+    int rows = TREE_ROWS;  // token rows the context's buffers hold: 64 * ceil(max_tree_nodes / 64), at most MAX_T
     int Hkv = 0;  // key/value heads: m.n_kv_heads, or m.n_heads when that is 0 (ordinary multi-head attention)
     cudaStream_t stream = nullptr;
     bool own_stream = false;
@@ -61,7 +62,7 @@ struct medusa_ctx {
     // test hooks for the bounded device-side waits (MEDUSA_OPT_SPIN_LIMIT, MEDUSA_OPT_WITHHOLD_LOAD)
     // (tile, k block) pairs per projection CTA that the kernel in front of a projection pulls into the L2 (prefetch.cuh);
     // 0 = off (MEDUSA_OPT_WEIGHT_PREFETCH)
-    int prefetch_units = 8;
+    int prefetch_units = 0;
     uint32_t spin_limit = 0;  // 0: the kernels' default
     int withhold = 0;         // one-shot: 1 = next tensor-core GEMM launch, 2 = next tcgen05 attention launch
     // host-side upper bound of the device-resident cache length (a hint for attention kernels that size their
@@ -73,7 +74,7 @@ struct medusa_ctx {
     bool use_tc = false;
     TensorMap map_xn, map_att, map_act, map_hidden, map_lm;
     std::vector<TensorMap> wmaps;  // per layer: wq, wk, wv, wo, w_gate, w_up, w_down
-    void *lo(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 ? (char *)hi + (size_t)TREE_ROWS * width * 2 : nullptr; }
+    void *lo(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 ? (char *)hi + (size_t)rows * width * 2 : nullptr; }
     float *logits = nullptr, *head_logits = nullptr;
     float2 *rope_cs = nullptr;
     void *tree_k = nullptr, *tree_v = nullptr, *k_cache = nullptr, *v_cache = nullptr;
@@ -225,7 +226,7 @@ struct ProfScope {
 // Tree attention of one layer: tensor-core flash kernel for bf16 / head_dim 128, CUDA-core kernel otherwise.
 int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v_new, const void *kc, const void *vc,
                   const int32_t *cache_len, const uint64_t *mask, void *out, void *out_lo, float *lse, int T, int L_hint,
-                  bool in_step, const void *q_lo = nullptr, const WeightPrefetch *pf = nullptr)
+                  bool in_step, int mask_words, const void *q_lo = nullptr, const WeightPrefetch *pf = nullptr)
 {
     const medusa_model_desc &m = c->m;
     if (c->flash_ws) {
@@ -233,7 +234,8 @@ int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v
         // Stand-alone, the tcgen05 kernel is the faster one from ATTN_TC_MIN_L cached keys on.  Inside a decode step it
         // is not: it fills the SM's shared and tensor memory, so the projection that follows cannot stream its first
         // weight tiles while the attention runs (measured at 7B width up to 3860 keys).
-        if (c->attn_mode == 2 || (c->attn_mode == 0 && !in_step && L_hint >= ATTN_TC_MIN_L))
+        // (the tcgen05 kernel holds one tile of 64 query rows: larger trees always take the mma.sync kernel)
+        if (T <= TREE_ROWS && (c->attn_mode == 2 || (c->attn_mode == 0 && !in_step && L_hint >= ATTN_TC_MIN_L)))
         {
             const int wh = c->withhold == 2 ? 1 : 0;
             if (wh) c->withhold = 0;
@@ -243,12 +245,12 @@ int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v
         }
         else
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_flash(q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse,
-                                                                     c->flash_ws, T, m.n_heads, c->Hkv, m.L_max, L_hint, c->stream, q_lo, pf));
+                                                                     c->flash_ws, T, m.n_heads, c->Hkv, m.L_max, L_hint, c->stream, q_lo, pf, mask_words));
         if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "flash attention launch failed: %s", cudaGetErrorString(e));
         return MEDUSA_OK;
     }
     PROF(c, PC_ATTENTION, 1, launch_tree_attention_simt(m.dtype, q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse, T,
-                                                        m.n_heads, c->Hkv, m.head_dim, m.L_max, c->stream));
+                                                        m.n_heads, c->Hkv, m.head_dim, m.L_max, c->stream, mask_words));
     MEDUSA_LAUNCH_CHECK(c);
     return MEDUSA_OK;
 }
@@ -267,12 +269,17 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
         *pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, (long long)plane_stride, seg0_cols);
         if (!whole_tiles && (size_t)pd->n_max * plane_stride > c->part_elems)
             return fail(c, MEDUSA_ERR_SHAPE, "projection needs %d partial planes, more than the workspace holds", pd->n_max);
-        cudaError_t e = cudaSuccess;
-        const int wh = c->withhold == 1 ? 1 : 0;
-        if (wh) c->withhold = 0;
-        PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, n_seg, seg_cols, K, *pd, P, ldy, T, row0, c->d_state + ST_STATUS,
-                                               c->stream, seg0_cols, c->spin_limit, wh));
-        if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "tensor-core GEMM launch failed: %s", cudaGetErrorString(e));
+        // the kernel covers 64 token rows: a larger tree is projected tile by tile (one launch per 64 rows, the weights
+        // streamed once per tile), every tile with the same plan, so the consumer finds the same pieces in every row
+        for (int r0 = (row0 / TREE_ROWS) * TREE_ROWS; r0 < T; r0 += TREE_ROWS) {
+            cudaError_t e = cudaSuccess;
+            const int wh = c->withhold == 1 ? 1 : 0;
+            if (wh) c->withhold = 0;
+            const int Tt = T - r0 < TREE_ROWS ? T - r0 : TREE_ROWS, row0t = row0 > r0 ? row0 - r0 : 0;
+            PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, n_seg, seg_cols, K, *pd, P + (size_t)r0 * ldy, ldy, Tt, row0t,
+                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0));
+            if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "tensor-core GEMM launch failed: %s", cudaGetErrorString(e));
+        }
         return MEDUSA_OK;
     }
     const char *Xr = (const char *)X + (size_t)row0 * K * c->esz;
@@ -290,7 +297,8 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
 
 // One backbone pass over T token rows (paper App. G Table 5, "parallel decoding" column).
 // logits are produced for rows [lm_row0, T).
-int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *mask, const int32_t *pos, int lm_row0)
+int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *mask, const int32_t *pos, int lm_row0,
+                  int mask_words)
 {
     const medusa_model_desc &m = c->m;
     const int d = m.d, H = m.n_heads, Hkv = c->Hkv, D = m.head_dim, HD = H * D, HkvD = Hkv * D, F = m.ffn, dt = m.dtype;
@@ -313,8 +321,8 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
         const WeightPrefetch pf_gu = gemm_tc_prefetch_plan(w_gu, 2, F, d, false, F, pfu);
         const WeightPrefetch pf_dn = gemm_tc_prefetch_plan(w_dn, 1, d, F, false, d, pfu);
         const TensorMap *wm = c->use_tc ? c->wmaps.data() + (size_t)l * 7 : nullptr;
-        char *tk = (char *)c->tree_k + (size_t)l * TREE_ROWS * HkvD * c->esz;
-        char *tv = (char *)c->tree_v + (size_t)l * TREE_ROWS * HkvD * c->esz;
+        char *tk = (char *)c->tree_k + (size_t)l * c->rows * HkvD * c->esz;
+        char *tv = (char *)c->tree_v + (size_t)l * c->rows * HkvD * c->esz;
         const char *kc = (const char *)c->k_cache + (size_t)l * Hkv * m.L_max * D * c->esz;
         const char *vc = (const char *)c->v_cache + (size_t)l * Hkv * m.L_max * D * c->esz;
         PlaneDesc pd{};
@@ -324,51 +332,51 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
         if (c->tap_layer >= 0) {
             const size_t planes = dt == MEDUSA_BF16 ? 2 : 1;
             if (l == c->tap_layer)
-                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_in, c->x, (size_t)TREE_ROWS * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_in, c->x, (size_t)c->rows * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
             if (l == c->tap_layer + 1) {
-                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)TREE_ROWS * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
-                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->xn, planes * TREE_ROWS * d * c->esz, cudaMemcpyDeviceToDevice, s));
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)c->rows * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->xn, planes * c->rows * d * c->esz, cudaMemcpyDeviceToDevice, s));
             }
         }
         const void *wqkv[3] = {w[1], w[2], w[3]};
         if (Hkv == H || !c->use_tc || (HD % 128 == 0 && HkvD % 128 == 0)) {
             // one launch for [q | k | v]; with grouped-query attention the k and v matrices are narrower than q
-            TRY(project(c, c->xn, &c->map_xn, wqkv, wm, 3, HkvD, d, c->part, (size_t)TREE_ROWS * qkv_ld, qkv_ld, T, 0, false, &pd, HD));
+            TRY(project(c, c->xn, &c->map_xn, wqkv, wm, 3, HkvD, d, c->part, (size_t)c->rows * qkv_ld, qkv_ld, T, 0, false, &pd, HD));
             PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd, 0, c->rope_cs, c->q, c->lo(c->q, HD), tk, tv, T, H, Hkv, D, s));
         } else {
             // widths that are not multiples of the 128-row tile: q alone (any width), then k and v on the CUDA-core
             // kernel, into disjoint columns of the same rows
             PlaneDesc pd_kv{};
-            TRY(project(c, c->xn, &c->map_xn, wqkv, wm, 1, HD, d, c->part, (size_t)TREE_ROWS * qkv_ld, qkv_ld, T, 0, false, &pd));
-            TRY(project(c, c->xn, &c->map_xn, wqkv + 1, wm ? wm + 1 : nullptr, 2, HkvD, d, c->part + HD, (size_t)TREE_ROWS * qkv_ld,
+            TRY(project(c, c->xn, &c->map_xn, wqkv, wm, 1, HD, d, c->part, (size_t)c->rows * qkv_ld, qkv_ld, T, 0, false, &pd));
+            TRY(project(c, c->xn, &c->map_xn, wqkv + 1, wm ? wm + 1 : nullptr, 2, HkvD, d, c->part + HD, (size_t)c->rows * qkv_ld,
                         qkv_ld, T, 0, false, &pd_kv));
             PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd_kv, HD, c->rope_cs, c->q, c->lo(c->q, HD), tk, tv, T, H, Hkv, D, s));
         }
         MEDUSA_LAUNCH_CHECK(c);
         TRY(attention(c, c->q, tk, tv, kc, vc, cache_len, mask, c->att, c->lo(c->att, HD), nullptr, T, c->L_upper, true,
-                      c->lo(c->q, HD), &pf_o));
+                      mask_words, c->lo(c->q, HD), &pf_o));
         if (l == c->tap_layer)
-            MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_att, c->att, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)TREE_ROWS * HD * c->esz,
+            MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_att, c->att, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)c->rows * HD * c->esz,
                                            cudaMemcpyDeviceToDevice, s));
         const void *wo[1] = {w[4]};
-        TRY(project(c, c->att, &c->map_att, wo, wm ? wm + 3 : nullptr, 1, d, HD, c->part, (size_t)TREE_ROWS * d, d, T, 0, false, &pd));
+        TRY(project(c, c->att, &c->map_att, wo, wm ? wm + 3 : nullptr, 1, d, HD, c->part, (size_t)c->rows * d, d, T, 0, false, &pd));
         // x += attention output projection;  xn = RMSNorm(x)
         PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd, w[5], m.rms_eps, c->xn, c->lo(c->xn, d), nullptr, T, d, s,
                                                    &pf_gu));
         const void *wgu[2] = {w[6], w[7]};
-        TRY(project(c, c->xn, &c->map_xn, wgu, wm ? wm + 4 : nullptr, 2, F, d, c->part, (size_t)TREE_ROWS * 2 * F, 2 * F, T, 0, false, &pd));
+        TRY(project(c, c->xn, &c->map_xn, wgu, wm ? wm + 4 : nullptr, 2, F, d, c->part, (size_t)c->rows * 2 * F, 2 * F, T, 0, false, &pd));
         PROF(c, PC_ELEMWISE, 1, launch_silu_mul(dt, c->part, pd, c->act, c->lo(c->act, F), T, F, s, &pf_dn));
         MEDUSA_LAUNCH_CHECK(c);
         const void *wd[1] = {w[8]};
-        TRY(project(c, c->act, &c->map_act, wd, wm ? wm + 6 : nullptr, 1, d, F, c->part, (size_t)TREE_ROWS * d, d, T, 0, false, &pd_prev));
+        TRY(project(c, c->act, &c->map_act, wd, wm ? wm + 6 : nullptr, 1, d, F, c->part, (size_t)c->rows * d, d, T, 0, false, &pd_prev));
     }
     const void *w_lm[3] = {c->w.lm_head, c->w.lm_head, c->w.lm_head};
     const WeightPrefetch pf_lm = gemm_tc_prefetch_plan(w_lm, 1, m.vocab, d, true, m.vocab, c->use_tc && d % 128 == 0 ? c->prefetch_units : 0);
     PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd_prev, c->w.final_norm, m.rms_eps, c->hidden,
                                                c->lo(c->hidden, d), c->hidden_f32, T, d, s, &pf_lm));
     if (c->tap_layer >= 0 && c->tap_layer == m.n_layers - 1) {
-        MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)TREE_ROWS * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
-        MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->hidden, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)TREE_ROWS * d * c->esz,
+        MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)c->rows * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+        MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->hidden, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)c->rows * d * c->esz,
                                        cudaMemcpyDeviceToDevice, s));
     }
     MEDUSA_LAUNCH_CHECK(c);
@@ -402,6 +410,8 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     if (m.dtype != MEDUSA_F32 && m.dtype != MEDUSA_BF16) return MEDUSA_ERR_INVALID_ARG;
     if (m.n_layers < 0 || m.d < 1 || m.n_heads < 1 || m.ffn < 1 || m.vocab < 1 || m.n_medusa < 0 || m.L_max < 0)
         return MEDUSA_ERR_INVALID_ARG;
+    if (m.max_tree_nodes < 0 || m.max_tree_nodes > MAX_T)
+        return MEDUSA_ERR_SHAPE;  // trees of up to MAX_T nodes
     if (m.n_kv_heads < 0 || (m.n_kv_heads > 0 && m.n_heads % m.n_kv_heads != 0))
         return MEDUSA_ERR_SHAPE;  // every key/value head serves the same number of query heads
     const int vn = m.dtype == MEDUSA_BF16 ? 8 : 4;
@@ -416,6 +426,7 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     if (!c) return MEDUSA_ERR_CUDA;
     c->m = m;
     c->device = device;
+    c->rows = m.max_tree_nodes <= TREE_ROWS ? TREE_ROWS : ((m.max_tree_nodes + TREE_ROWS - 1) / TREE_ROWS) * TREE_ROWS;
     c->stream = (cudaStream_t)stream;
     if (!c->stream) {
         // The legacy default stream cannot be captured into a graph.  A blocking stream orders itself with the
@@ -431,9 +442,9 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     MEDUSA_CUDA(c, cudaSetDevice(device));
     c->Hkv = m.n_kv_heads > 0 ? m.n_kv_heads : m.n_heads;
     const size_t d = m.d, HD = (size_t)m.n_heads * m.head_dim, HkvD = (size_t)c->Hkv * m.head_dim, F = m.ffn, V = m.vocab,
-                 K = m.n_medusa, R = TREE_ROWS;
+                 K = m.n_medusa, R = (size_t)c->rows;
     TRY(dev_alloc(c, &c->d_state, ST_WORDS));
-    TRY(dev_alloc(c, &c->d_mask, R));
+    TRY(dev_alloc(c, &c->d_mask, R * (R / 64)));
     TRY(dev_alloc(c, &c->d_chain_mask, R));
     TRY(dev_alloc(c, &c->d_pos, R));
     TRY(dev_alloc(c, &c->d_chain_pos, R));
@@ -471,7 +482,7 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     TRY(dev_alloc_bytes(c, &c->tap_att, planes * R * HD * c->esz));
     TRY(dev_alloc_bytes(c, &c->tap_xn_out, planes * R * d * c->esz));
     if (m.dtype == MEDUSA_BF16 && m.head_dim == 128 && tuning_env("MEDUSA_FORCE_SIMT_ATTENTION") == nullptr)
-        TRY(dev_alloc_bytes(c, &c->flash_ws, tree_attention_flash_workspace_bytes(m.n_heads)));
+        TRY(dev_alloc_bytes(c, &c->flash_ws, tree_attention_flash_workspace_bytes(m.n_heads, c->rows / TREE_ROWS)));
     if (const char *e = tuning_env("MEDUSA_ATTENTION"))
         c->attn_mode = strcmp(e, "tcgen05") == 0 ? 2 : (strcmp(e, "mma_sync") == 0 ? 1 : 0);
     c->use_tc = m.dtype == MEDUSA_BF16 && tuning_env("MEDUSA_FORCE_SIMT_GEMM") == nullptr && !(d % 8 || HD % 8 || HkvD % 8 || F % 8);
@@ -498,8 +509,8 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
         TRY(dev_alloc(c, &c->part, R * need));
     }
     if (c->use_tc) {
-        if (!make_act_map(&c->map_xn, c->xn, (int)d) || !make_act_map(&c->map_att, c->att, (int)HD) ||
-            !make_act_map(&c->map_act, c->act, (int)F) || !make_act_map(&c->map_hidden, c->hidden, (int)d))
+        if (!make_act_map(&c->map_xn, c->xn, (int)d, c->rows) || !make_act_map(&c->map_att, c->att, (int)HD, c->rows) ||
+            !make_act_map(&c->map_act, c->act, (int)F, c->rows) || !make_act_map(&c->map_hidden, c->hidden, (int)d, c->rows))
             return fail(c, MEDUSA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the activation planes");
     }
     PROF(c, PC_ELEMWISE,1, launch_iota(c->iota, (int)R, c->stream));
@@ -513,7 +524,7 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     }
     MEDUSA_CUDA(c, cudaMemcpyAsync(c->d_chain_mask, cm, sizeof cm, cudaMemcpyHostToDevice, c->stream));
     MEDUSA_CUDA(c, cudaMemcpyAsync(c->d_chain_pos, cp, sizeof cp, cudaMemcpyHostToDevice, c->stream));
-    MEDUSA_CUDA(c, cudaHostAlloc((void **)&c->pinned, (TREE_ROWS + 8) * sizeof(int32_t), cudaHostAllocDefault));
+    MEDUSA_CUDA(c, cudaHostAlloc((void **)&c->pinned, (TREE_ROWS + 8) * sizeof(int32_t), cudaHostAllocDefault));  // depth + 1 <= 9 tokens per step
     MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
     return MEDUSA_OK;
 }
@@ -557,7 +568,7 @@ static void drop_step_graphs(medusa_ctx *c)
 static const void *workspace_view(medusa_ctx *c, int32_t which, size_t *bytes)
 {
     const medusa_model_desc &m = c->m;
-    const size_t R = TREE_ROWS, d = m.d, V = m.vocab, K = m.n_medusa ? m.n_medusa : 1, HD = (size_t)m.n_heads * m.head_dim;
+    const size_t R = (size_t)c->rows, d = m.d, V = m.vocab, K = m.n_medusa ? m.n_medusa : 1, HD = (size_t)m.n_heads * m.head_dim;
     const size_t HkvD = (size_t)c->Hkv * m.head_dim, planes = m.dtype == MEDUSA_BF16 ? 2 : 1;
     const size_t cache_bytes = (size_t)m.n_layers * HkvD * m.L_max * c->esz, tree_bytes = (size_t)m.n_layers * R * HkvD * c->esz;
     const void *p = nullptr;
@@ -723,11 +734,14 @@ extern "C" int32_t medusa_build_tree_buffers(medusa_ctx *c, const int32_t *paths
 {
     TreeHost tr;
     int32_t rc = build_tree(paths_host, n_paths, max_depth, tr);
-    if (rc != MEDUSA_OK) return fail(c, rc, "invalid tree: tuples must be distinct, prefix-closed, -1 padded, T <= 64");
+    if (rc != MEDUSA_OK) return fail(c, rc, "invalid tree: tuples must be distinct, prefix-closed, -1 padded, T <= %d", MAX_T);
     if (c && tr.depth > c->m.n_medusa) return fail(c, MEDUSA_ERR_SHAPE, "tree depth %d exceeds the %d Medusa heads", tr.depth, c->m.n_medusa);
+    if (c && tr.T > c->rows)
+        return fail(c, MEDUSA_ERR_SHAPE, "a tree of %d nodes does not fit this context (created for trees of up to %d nodes: "
+                    "set max_tree_nodes in the model descriptor)", tr.T, c->rows);
     if (out) {
         out->T = tr.T; out->P = tr.P; out->depth = tr.depth; out->topk = tr.topk;
-        if (out->mask) memcpy(out->mask, tr.mask.data(), tr.T * sizeof(uint64_t));
+        if (out->mask) memcpy(out->mask, tr.mask.data(), tr.mask.size() * sizeof(uint64_t));
         if (out->pos) memcpy(out->pos, tr.pos.data(), tr.T * sizeof(int32_t));
         if (out->tree_idx) memcpy(out->tree_idx, tr.tree_idx.data(), tr.T * sizeof(int32_t));
         if (out->parent) memcpy(out->parent, tr.parent.data(), tr.T * sizeof(int32_t));
@@ -736,7 +750,7 @@ extern "C" int32_t medusa_build_tree_buffers(medusa_ctx *c, const int32_t *paths
     if (c) {
         MEDUSA_CUDA(c, cudaSetDevice(c->device));
         MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));  // earlier work may still read the old tree
-        MEDUSA_CUDA(c, cudaMemcpy(c->d_mask, tr.mask.data(), tr.T * sizeof(uint64_t), cudaMemcpyHostToDevice));
+        MEDUSA_CUDA(c, cudaMemcpy(c->d_mask, tr.mask.data(), tr.mask.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
         MEDUSA_CUDA(c, cudaMemcpy(c->d_pos, tr.pos.data(), tr.T * sizeof(int32_t), cudaMemcpyHostToDevice));
         MEDUSA_CUDA(c, cudaMemcpy(c->d_tree_idx, tr.tree_idx.data(), tr.T * sizeof(int32_t), cudaMemcpyHostToDevice));
         MEDUSA_CUDA(c, cudaMemcpy(c->d_parent, tr.parent.data(), tr.T * sizeof(int32_t), cudaMemcpyHostToDevice));
@@ -805,7 +819,7 @@ extern "C" int32_t medusa_tree_attention(medusa_ctx *c, const void *q, const voi
     // the cache length lives on the device here: the kernel choice and the tcgen05 kernel's grid follow the caller's
     // bound (MEDUSA_OPT_ATTENTION_LENGTH_HINT), or the full capacity if none was given
     const int hint = c->attn_len_hint < 0 || c->attn_len_hint > m.L_max ? m.L_max : c->attn_len_hint;
-    return attention(c, qq, kk, v_new, k_cache, v_cache, cache_len, c->d_mask, out, nullptr, lse, T, hint, false);
+    return attention(c, qq, kk, v_new, k_cache, v_cache, cache_len, c->d_mask, out, nullptr, lse, T, hint, false, c->tree.mask_words);
 }
 
 // ============================================================================ a7: acceptance
@@ -852,7 +866,7 @@ extern "C" int32_t medusa_accept_and_update_kv(medusa_ctx *c, const void *tree_k
     a.accept_len = accept_len; a.max_commit = max_commit; a.cache_len = cache_len; a.hidden = hidden; a.h_last = h_last;
     a.tree_tok = tree_tok; a.emitted = emitted; a.n_emitted = n_emitted; a.status = c->d_state + ST_STATUS;
     a.next_root = nullptr; a.root_out = nullptr;
-    a.n_layers = c->m.n_layers; a.H = c->Hkv; a.D = c->m.head_dim; a.L_max = c->m.L_max; a.d = c->m.d;
+    a.tree_rows = c->rows; a.n_layers = c->m.n_layers; a.H = c->Hkv; a.D = c->m.head_dim; a.L_max = c->m.L_max; a.d = c->m.d;
     a.depth_plus1 = c->tree.depth + 1;
     PROF(c, PC_COMMIT,2, launch_commit(c->m.dtype, a, c->stream));
     MEDUSA_LAUNCH_CHECK(c);
@@ -878,7 +892,7 @@ extern "C" int32_t medusa_load_weights(medusa_ctx *c, const medusa_weights *w)
     if (!c->k_cache) {
         const size_t HkvD = (size_t)c->Hkv * m.head_dim;
         const size_t cache_bytes = (size_t)m.n_layers * HkvD * m.L_max * c->esz;
-        const size_t tree_bytes = (size_t)m.n_layers * TREE_ROWS * HkvD * c->esz;
+        const size_t tree_bytes = (size_t)m.n_layers * c->rows * HkvD * c->esz;
         TRY(dev_alloc_bytes(c, &c->k_cache, cache_bytes));
         TRY(dev_alloc_bytes(c, &c->v_cache, cache_bytes));
         TRY(dev_alloc_bytes(c, &c->tree_k, tree_bytes));
@@ -919,7 +933,7 @@ static int32_t prefill_dev(medusa_ctx *c, const int32_t *prompt, int32_t n, int3
     if (L0 + n > m.L_max) return fail(c, MEDUSA_ERR_CACHE_FULL, "prompt of %d tokens does not fit the cache (L_max %d)", n, m.L_max);
     for (int off = 0; off < n; off += TREE_ROWS) {
         const int T = n - off < TREE_ROWS ? n - off : TREE_ROWS;
-        TRY(tree_pass(c, prompt + off, T, c->d_chain_mask, c->d_chain_pos, T - 1));
+        TRY(tree_pass(c, prompt + off, T, c->d_chain_mask, c->d_chain_pos, T - 1, 1));
         PROF(c, PC_ELEMWISE, 1, (launch_pdl(set_i32_kernel, dim3(1), dim3(1), 0, c->stream, c->tmp_i32, T - 1)));  // "accept_len" of a chain: everything
         PROF(c, PC_POSTERIOR,1, launch_argmax_row(c->logits, m.vocab, T - 1, c->tmp_i32 + 1, c->stream));
         CommitArgs a{};
@@ -928,7 +942,7 @@ static int32_t prefill_dev(medusa_ctx *c, const int32_t *prompt, int32_t n, int3
         a.hidden = c->hidden_f32; a.h_last = c->h_last; a.tree_tok = prompt + off; a.emitted = c->emitted;
         a.n_emitted = c->d_state + ST_N_EMITTED; a.status = c->d_state + ST_STATUS;
         a.next_root = c->tmp_i32 + 1; a.root_out = c->d_state + ST_ROOT;
-        a.n_layers = m.n_layers; a.H = c->Hkv; a.D = m.head_dim; a.L_max = m.L_max; a.d = m.d; a.depth_plus1 = T;
+        a.tree_rows = c->rows; a.n_layers = m.n_layers; a.H = c->Hkv; a.D = m.head_dim; a.L_max = m.L_max; a.d = m.d; a.depth_plus1 = T;
         PROF(c, PC_COMMIT,2, launch_commit(m.dtype, a, c->stream));
         MEDUSA_LAUNCH_CHECK(c);
         c->L_upper += T;
@@ -953,7 +967,7 @@ extern "C" int32_t medusa_tree_pass(medusa_ctx *c, const int32_t *tokens)
     TRY(check_ready(c, true, true));
     if (!tokens) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_tree_pass: null tokens");
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
-    return tree_pass(c, tokens, c->tree.T, c->d_mask, c->d_pos, 0);
+    return tree_pass(c, tokens, c->tree.T, c->d_mask, c->d_pos, 0, c->tree.mask_words);
 }
 
 // Everything one decode step enqueues on the context's stream (no host-side state is touched).
@@ -965,7 +979,7 @@ static int32_t decode_step_launches(medusa_ctx *c, const medusa_accept_params *p
     // (1) candidates: heads on the last accepted hidden state, top-k, tree tokens
     TRY(heads_impl(c, c->h_last, 1, c->w.medusa_w1, c->w.medusa_w2, st + ST_ROOT, c->topk_idx, nullptr, nullptr, c->tree_tok));
     // (2) process them: one backbone pass with tree attention
-    TRY(tree_pass(c, c->tree_tok, c->tree.T, c->d_mask, c->d_pos, 0));
+    TRY(tree_pass(c, c->tree_tok, c->tree.T, c->d_mask, c->d_pos, 0, c->tree.mask_words));
     // (3) accept: longest accepted prefix, then commit its K/V
     TRY(medusa_evaluate_posterior(c, c->logits, c->tree_tok, params, gumbel, st + ST_BEST, st + ST_ACCEPT_LEN,
                                   st + ST_NEXT_ROOT, c->acc_nodes));
@@ -975,7 +989,7 @@ static int32_t decode_step_launches(medusa_ctx *c, const medusa_accept_params *p
     a.cache_len = st + ST_CACHE_LEN; a.hidden = c->hidden_f32; a.h_last = c->h_last; a.tree_tok = c->tree_tok;
     a.emitted = c->emitted; a.n_emitted = st + ST_N_EMITTED; a.status = st + ST_STATUS;
     a.next_root = st + ST_NEXT_ROOT; a.root_out = st + ST_ROOT;
-    a.n_layers = m.n_layers; a.H = c->Hkv; a.D = m.head_dim; a.L_max = m.L_max; a.d = m.d;
+    a.tree_rows = c->rows; a.n_layers = m.n_layers; a.H = c->Hkv; a.D = m.head_dim; a.L_max = m.L_max; a.d = m.d;
     a.depth_plus1 = c->tree.depth + 1;
     PROF(c, PC_COMMIT,2, launch_commit(m.dtype, a, c->stream));
     MEDUSA_LAUNCH_CHECK(c);

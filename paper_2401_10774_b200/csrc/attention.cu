@@ -15,7 +15,7 @@ tree_attention_simt_kernel(const AT *__restrict__ q, const AT *__restrict__ k_ne
                            const AT *__restrict__ k_cache, const AT *__restrict__ v_cache,
                            const int32_t *__restrict__ cache_len, const uint64_t *__restrict__ mask,
                            AT *__restrict__ out, AT *__restrict__ out_lo, float *__restrict__ lse, int T, int H,
-                           int Hkv, int L_max)
+                           int Hkv, int L_max, int mask_words)
 {
     pdl_enter();
     constexpr int E = D / 32;  // elements per lane
@@ -33,7 +33,7 @@ tree_attention_simt_kernel(const AT *__restrict__ q, const AT *__restrict__ k_ne
         o[e] = 0.f;
     }
     float m = -INFINITY, l = 0.f;
-    const uint64_t mk = mask[i];
+    const uint64_t *mk = mask + (size_t)i * mask_words;  // the query's ancestor set, 64 tree nodes per word
     const int nk = L + T;
     for (int j = 0; j < nk; ++j) {
         const AT *kp, *vp;
@@ -41,7 +41,7 @@ tree_attention_simt_kernel(const AT *__restrict__ q, const AT *__restrict__ k_ne
             kp = k_cache + ((size_t)hk * L_max + j) * D;
             vp = v_cache + ((size_t)hk * L_max + j) * D;
         } else {
-            if (!((mk >> (j - L)) & 1ull))
+            if (!((mk[(j - L) >> 6] >> ((j - L) & 63)) & 1ull))
                 continue;
             kp = k_new + ((size_t)(j - L) * Hkv + hk) * D;
             vp = v_new + ((size_t)(j - L) * Hkv + hk) * D;
@@ -75,13 +75,14 @@ tree_attention_simt_kernel(const AT *__restrict__ q, const AT *__restrict__ k_ne
 
 void launch_tree_attention_simt(int dtype, const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                 const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
-                                void *out_lo, float *lse, int T, int H, int Hkv, int D, int L_max, cudaStream_t s)
+                                void *out_lo, float *lse, int T, int H, int Hkv, int D, int L_max, cudaStream_t s,
+                                int mask_words)
 {
     dim3 grid((T + 3) / 4, H);
 #define MEDUSA_ATT(AT, DD)                                                                                         \
     launch_pdl(tree_attention_simt_kernel<AT, DD>, dim3(grid), dim3(128), 0, s, (const AT *)q, (const AT *)k_new, (const AT *)v_new,  \
                                                             (const AT *)k_cache, (const AT *)v_cache, cache_len,  \
-                                                            mask, (AT *)out, (AT *)out_lo, lse, T, H, Hkv, L_max)
+                                                            mask, (AT *)out, (AT *)out_lo, lse, T, H, Hkv, L_max, mask_words)
     if (dtype == MEDUSA_BF16) {
         if (D == 128) MEDUSA_ATT(bf16, 128); else MEDUSA_ATT(bf16, 64);
     } else {

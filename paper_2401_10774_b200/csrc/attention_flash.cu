@@ -28,19 +28,7 @@ namespace {
 constexpr int D = 128;          // head dim
 constexpr int BQ = 64;          // query rows per CTA (4 warps x 16)
 constexpr int BKEY = 64;        // keys per tile
-#ifndef ATT_STAGES
-#define ATT_STAGES 3
-#endif
-#ifndef ATT_PREFETCH
-#define ATT_PREFETCH 1
-#endif
-#ifndef ATT_RANGES
-#define ATT_RANGES 1
-#endif
-#ifndef ATT_QLO
-#define ATT_QLO 1
-#endif
-constexpr int STAGES = ATT_STAGES;
+constexpr int STAGES = 3;
 constexpr int THREADS = 256;     // 8 warps: warp w owns query rows 16*(w&3).. and key half (w>>2) of every tile
 constexpr int TILE_BYTES = BKEY * D * 2;           // 16 KiB for K, same for V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
@@ -88,12 +76,14 @@ struct Args {
     const bf16 *q_lo;                // nullable [T][H][D]: second plane of q (scores are q.k + q_lo.k)
     const bf16 *k_cache, *v_cache;   // [H][L_max][D]
     const int32_t *cache_len;
-    const uint64_t *mask;            // [T]
+    const uint64_t *mask;            // [T][mask_words]: bit j of row i -- tree node j visible to query i
+    int mask_words;                  // 64 tree nodes per word
+    int q_tiles;                     // tiles of 64 query rows (gridDim.z); a query tile sees the tree's key tiles 0..its own
     bf16 *out, *out_lo;              // [T][H][D]; out_lo nullable
     float *lse;                      // nullable [T][H]
-    float *ws_o;                     // [H][max_splits][64][128] unnormalised partial outputs
-    float *ws_ml;                    // [H][max_splits][2][64]  running max (log2 domain) and sum
-    int *counters;                   // [H] arrival tickets, zero between launches
+    float *ws_o;                     // [q_tiles][H][max_splits][64][128] unnormalised partial outputs
+    float *ws_ml;                    // [q_tiles][H][max_splits][2][64]  running max (log2 domain) and sum
+    int *counters;                   // [q_tiles][H] arrival tickets, zero between launches
     int T, H, L_max, tiles_per_split, max_splits;
     int Hkv;                         // key/value heads; query head h reads key/value head h / (H / Hkv)
     int rows_max_tiles;              // caches of up to this many tiles run in row-split mode (0: never)
@@ -355,20 +345,14 @@ __device__ __forceinline__ Ranges plan_ranges(const Args &a, int L_raw, int sp)
     // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
     r.L = min(max(L_raw, 0), a.L_max);
     r.nt = (r.L + BKEY - 1) / BKEY;
-    r.rows_mode = r.nt <= a.rows_max_tiles && gridDim.y >= 2;
+    r.rows_mode = r.nt <= a.rows_max_tiles && gridDim.y >= 2 && a.q_tiles == 1;
     // Key ranges: fixed by the launch (tiles_per_split > 0), or chosen here from the true cache length, so that the
     // result does not depend on what the host knew about the length when it launched: as many ranges as the grid has
     // rows (one wave of CTAs; every CTA requests its first tiles before the dependency wait, so a range costs little
     // to start), but no range shorter than two tiles.
     int tps = a.tiles_per_split;
     if (tps <= 0) {
-#if ATT_RANGES == 1
         const int want = min((int)gridDim.y, max(1, r.nt / 2));
-#else
-        int want = 1;
-        while (want * want < r.nt) ++want;
-        want = min(want, (int)gridDim.y);
-#endif
         tps = r.nt > 0 ? (r.nt + want - 1) / want : 1;
     }
     const int n_cache_splits = (r.nt + tps - 1) / tps;
@@ -379,7 +363,8 @@ __device__ __forceinline__ Ranges plan_ranges(const Args &a, int L_raw, int sp)
     r.tile0 = sp * tps;
     r.has_tree = sp == r.n_active - 1;
     r.tile1 = r.has_tree ? r.nt : min(r.nt, r.tile0 + tps);
-    r.n_tiles = (r.tile1 - r.tile0) + (r.has_tree ? 1 : 0);
+    // the last range also takes the tree's own keys: query tile z needs the key tiles 0..z (ancestors come first)
+    r.n_tiles = (r.tile1 - r.tile0) + (r.has_tree ? (int)blockIdx.z + 1 : 0);
     return r;
 }
 
@@ -391,6 +376,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     const bool has_qlo = a.q_lo != nullptr;
     __shared__ int s_ticket;
     const int h = blockIdx.x, sp = blockIdx.y;
+    const int q0 = (int)blockIdx.z * BQ;      // first query row of this CTA's tile
+    const int Tq = min(BQ, a.T - q0);         // its query rows
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 3, kh = warp >> 2;  // query-row group, key half
     const size_t HD = (size_t)a.H * D, HkvD = (size_t)a.Hkv * D;
@@ -401,14 +388,9 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     // values, which are requested after the wait.  The length is read again after the wait; should it differ (never
     // observed), the prefetched tiles are dropped and requested again.
     Ranges rg = plan_ranges(a, *a.cache_len, sp);
-    bool waited = false;
     auto prefetch_cache_tiles = [&]() {
         if (rg.rows_mode || rg.idle)
             return;
-#if !ATT_PREFETCH
-        if (!waited)
-            return;
-#endif
         for (int i = 0; i < STAGES - 1; ++i) {
             const int ct = rg.tile0 + i;
             if (ct < rg.tile1) {
@@ -419,14 +401,9 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
         }
     };
     prefetch_cache_tiles();
-    prefetch_weights(a.pf, ((long long)blockIdx.y * gridDim.x + blockIdx.x) * THREADS + threadIdx.x,
-                     (long long)gridDim.x * gridDim.y * THREADS);
+    prefetch_weights(a.pf, (((long long)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * THREADS + threadIdx.x,
+                     (long long)gridDim.x * gridDim.y * gridDim.z * THREADS);
     pdl_wait();
-    waited = true;
-#if !ATT_PREFETCH
-    rg = plan_ranges(a, *a.cache_len, sp);
-    prefetch_cache_tiles();
-#endif
     {
         const int L_now = min(max(*a.cache_len, 0), a.L_max);
         if (L_now != rg.L) {
@@ -454,23 +431,26 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             const size_t base = ((size_t)hk * a.L_max + (size_t)ct * BKEY) * D;
             load_tile(stage, a.k_cache + base, a.v_cache + base, D, min(BKEY, L - ct * BKEY));
         } else {
-            load_tile(stage, a.k_new + (size_t)hk * D, a.v_new + (size_t)hk * D, HkvD, a.T);
+            const int w = ct - tile1;  // key tile of the tree
+            const size_t base = ((size_t)w * BKEY * a.Hkv + hk) * D;
+            load_tile(stage, a.k_new + base, a.v_new + base, HkvD, min(BKEY, a.T - w * BKEY));
         }
     };
-    // ---- after the wait: Q, and the tree's own tile if it is one of the first STAGES-1 tiles, as one more copy group
+    // ---- after the wait: Q, and the tree's own tiles that are among the first STAGES-1 tiles, as one more copy group
     {
         const uint32_t qb = smem_u32(smem_all);
 #pragma unroll
         for (int i = 0; i < 1024 / THREADS; ++i) {
             int idx = threadIdx.x + i * THREADS;
             int r = idx >> 4, c = idx & 15;
-            bool ok = r < a.T;
-            cp_async16(qb + tile_off(r, c), a.q + (size_t)(ok ? r : 0) * HD + (size_t)h * D + c * 8, ok);
+            bool ok = r < Tq;
+            cp_async16(qb + tile_off(r, c), a.q + (size_t)(ok ? q0 + r : 0) * HD + (size_t)h * D + c * 8, ok);
             if (has_qlo)
-                cp_async16(qb + TILE_BYTES + tile_off(r, c), a.q_lo + (size_t)(ok ? r : 0) * HD + (size_t)h * D + c * 8, ok);
+                cp_async16(qb + TILE_BYTES + tile_off(r, c), a.q_lo + (size_t)(ok ? q0 + r : 0) * HD + (size_t)h * D + c * 8, ok);
         }
-        if (rg.has_tree && n_tiles - 1 < STAGES - 1)
-            issue(n_tiles - 1);
+        for (int i = 0; i < STAGES - 1; ++i)
+            if (i < n_tiles && tile0 + i >= tile1)
+                issue(i);
         cp_async_commit();
     }
     cp_async_wait<0>();  // Q and the first STAGES-1 tiles have landed
@@ -485,8 +465,7 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             ldsm_x4(qb + tile_off(q_row, 2 * ks + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
     }
 
-    const int row0 = wq * 16 + g, row1 = row0 + 8;
-    const uint64_t mask0 = row0 < a.T ? a.mask[row0] : 0ull, mask1 = row1 < a.T ? a.mask[row1] : 0ull;
+    const int row0 = wq * 16 + g, row1 = row0 + 8;  // rows inside the query tile
     const float sc = rsqrtf((float)D) * LOG2E;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     float o[16][4];
@@ -530,6 +509,13 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
         // ---- mask + online softmax (log2 domain)
         float mx0 = -INFINITY, mx1 = -INFINITY;
         const int key_base = ct * BKEY;
+        // a tree tile: this thread's two query rows' mask words for that key tile (ancestors inside keys 64 w .. 64 w + 63)
+        uint64_t mask0 = 0ull, mask1 = 0ull;
+        if (tree_tile) {
+            const int w = ct - tile1;
+            if (row0 < Tq) mask0 = a.mask[(size_t)(q0 + row0) * a.mask_words + w];
+            if (row1 < Tq) mask1 = a.mask[(size_t)(q0 + row1) * a.mask_words + w];
+        }
 #pragma unroll
         for (int n = 0; n < 4; ++n) {
 #pragma unroll
@@ -641,8 +627,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
 #pragma unroll
         for (int dn = 0; dn < 16; ++dn) {
             const int col = dn * 8 + 2 * t4;
-            if (owner && row0 < a.T) {
-                const size_t idx = (size_t)row0 * HD + (size_t)h * D + col;
+            if (owner && row0 < Tq) {
+                const size_t idx = (size_t)(q0 + row0) * HD + (size_t)h * D + col;
                 const float y0 = o[dn][0] * i0, y1 = o[dn][1] * i0;
                 const __nv_bfloat162 hi = __floats2bfloat162_rn(y0, y1);
                 *reinterpret_cast<__nv_bfloat162 *>(a.out + idx) = hi;
@@ -650,8 +636,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
                     *reinterpret_cast<__nv_bfloat162 *>(a.out_lo + idx) =
                         __floats2bfloat162_rn(y0 - __low2float(hi), y1 - __high2float(hi));
             }
-            if (owner && row1 < a.T) {
-                const size_t idx = (size_t)row1 * HD + (size_t)h * D + col;
+            if (owner && row1 < Tq) {
+                const size_t idx = (size_t)(q0 + row1) * HD + (size_t)h * D + col;
                 const float y0 = o[dn][2] * i1, y1 = o[dn][3] * i1;
                 const __nv_bfloat162 hi = __floats2bfloat162_rn(y0, y1);
                 *reinterpret_cast<__nv_bfloat162 *>(a.out + idx) = hi;
@@ -661,14 +647,15 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             }
         }
         if (a.lse && t4 == 0 && owner) {
-            if (row0 < a.T) a.lse[(size_t)row0 * a.H + h] = m0 / LOG2E + logf(l0);
-            if (row1 < a.T) a.lse[(size_t)row1 * a.H + h] = m1 / LOG2E + logf(l1);
+            if (row0 < Tq) a.lse[(size_t)(q0 + row0) * a.H + h] = m0 / LOG2E + logf(l0);
+            if (row1 < Tq) a.lse[(size_t)(q0 + row1) * a.H + h] = m1 / LOG2E + logf(l1);
         }
         return;
     }
     // ---- partial result of this key range
-    float *wo = a.ws_o + ((size_t)h * a.max_splits + sp) * BQ * D;
-    float *wml = a.ws_ml + ((size_t)h * a.max_splits + sp) * 2 * BQ;
+    const size_t slot = (size_t)blockIdx.z * a.H + h;  // (query tile, head)
+    float *wo = a.ws_o + (slot * a.max_splits + sp) * BQ * D;
+    float *wml = a.ws_ml + (slot * a.max_splits + sp) * 2 * BQ;
     if (owner) {
 #pragma unroll
         for (int dn = 0; dn < 16; ++dn) {
@@ -685,7 +672,7 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0)
-        s_ticket = atomicAdd(a.counters + h, 1);
+        s_ticket = atomicAdd(a.counters + slot, 1);
     __syncthreads();
     if (s_ticket != n_active - 1)
         return;
@@ -694,8 +681,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     // transaction) together with the partial outputs, two ranges per round, all loads of a round in flight at once, and
     // folds them in with a running maximum: one trip to the L2 instead of a staged max / weight / output sequence.
     __threadfence();
-    const float *__restrict__ mlh = a.ws_ml + (size_t)h * a.max_splits * 2 * BQ;
-    const float *__restrict__ oh = a.ws_o + (size_t)h * a.max_splits * BQ * D;
+    const float *__restrict__ mlh = a.ws_ml + slot * a.max_splits * 2 * BQ;
+    const float *__restrict__ oh = a.ws_o + slot * a.max_splits * BQ * D;
     const int c4 = (threadIdx.x & 31) * 4, r8 = (threadIdx.x >> 5) * 8;
     float mrun[8], lrun[8];
     float4 acc[8];
@@ -752,11 +739,11 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
         const int r = r8 + u;
-        if (r >= a.T)
+        if (r >= Tq)
             continue;
         const float inv = lrun[u] > 0.f ? 1.0f / lrun[u] : 0.f;
         const float y[4] = {acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv};
-        const size_t idx = (size_t)r * HD + (size_t)h * D + c4;
+        const size_t idx = (size_t)(q0 + r) * HD + (size_t)h * D + c4;
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]), h1 = __floats2bfloat162_rn(y[2], y[3]);
         uint2 pk;
         pk.x = *reinterpret_cast<const uint32_t *>(&h0);
@@ -770,10 +757,10 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             *reinterpret_cast<uint2 *>(a.out_lo + idx) = pk;
         }
         if (a.lse && c4 == 0)
-            a.lse[(size_t)r * a.H + h] = mrun[u] / LOG2E + logf(lrun[u]);
+            a.lse[(size_t)(q0 + r) * a.H + h] = mrun[u] / LOG2E + logf(lrun[u]);
     }
     if (threadIdx.x == 0)
-        a.counters[h] = 0;  // ready for the next launch
+        a.counters[slot] = 0;  // ready for the next launch
 }
 
 }  // namespace
@@ -787,15 +774,16 @@ static int rows_mode_max_tiles()
 
 static bool g_flash_attr_set[64] = {};  // devices on which the kernel's shared-memory limit has been raised
 
-size_t tree_attention_flash_workspace_bytes(int H)
+size_t tree_attention_flash_workspace_bytes(int H, int q_tiles)
 {
-    return (size_t)H * FLASH_MAX_SPLITS * (BQ * D + 2 * BQ) * sizeof(float) + (size_t)H * sizeof(int);
+    const size_t slots = (size_t)H * (q_tiles > 0 ? q_tiles : 1);
+    return slots * FLASH_MAX_SPLITS * (BQ * D + 2 * BQ) * sizeof(float) + slots * sizeof(int);
 }
 
 cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                        int L_hint, cudaStream_t s, const void *q_lo, const WeightPrefetch *prefetch)
+                                        int L_hint, cudaStream_t s, const void *q_lo, const WeightPrefetch *prefetch, int mask_words)
 {
     if (first_use_on_current_device(g_flash_attr_set)) {
         cudaError_t e = cudaFuncSetAttribute(tree_attention_flash_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -818,16 +806,20 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
     }
     Args a;
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
-    a.q_lo = ATT_QLO ? (const bf16 *)q_lo : nullptr;
+    a.q_lo = (const bf16 *)q_lo;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
     a.cache_len = cache_len; a.mask = mask; a.out = (bf16 *)out; a.out_lo = (bf16 *)out_lo; a.lse = lse;
+    const int q_tiles = (T + BQ - 1) / BQ;
+    const size_t slots = (size_t)H * q_tiles;
     a.ws_o = (float *)workspace;
-    a.ws_ml = a.ws_o + (size_t)H * FLASH_MAX_SPLITS * BQ * D;
-    a.counters = (int *)(a.ws_ml + (size_t)H * FLASH_MAX_SPLITS * 2 * BQ);
+    a.ws_ml = a.ws_o + slots * FLASH_MAX_SPLITS * BQ * D;
+    a.counters = (int *)(a.ws_ml + slots * FLASH_MAX_SPLITS * 2 * BQ);
+    a.mask_words = mask_words > 0 ? mask_words : 1;
+    a.q_tiles = q_tiles;
     a.T = T; a.H = H; a.Hkv = Hkv; a.L_max = L_max; a.tiles_per_split = tps; a.max_splits = FLASH_MAX_SPLITS;
     a.rows_max_tiles = rows_mode_max_tiles();
     a.pf = prefetch ? *prefetch : WeightPrefetch{};
-    dim3 grid(H, splits);
+    dim3 grid(H, splits, q_tiles);
     launch_pdl(tree_attention_flash_kernel, dim3(grid), dim3(THREADS), SMEM_BYTES, s, a);
     return cudaGetLastError();
 }
@@ -921,6 +913,8 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
         tps = (nt + STATIC_MAX_SPLITS - 1) / STATIC_MAX_SPLITS;
         splits = (nt + tps - 1) / tps;
     }
+    a.mask_words = 1;
+    a.q_tiles = 1;
     a.T = T; a.H = H; a.Hkv = H; a.L_max = L_max; a.tiles_per_split = tps; a.max_splits = STATIC_MAX_SPLITS;
     a.rows_max_tiles = rows_mode_max_tiles();
     a.pf = WeightPrefetch{};

@@ -9,9 +9,11 @@
 
 namespace medusa {
 
-constexpr int MAX_T = 64;       // tree nodes incl. root (one 64-bit mask word per query)
+constexpr int MAX_T = 256;      // tree nodes incl. root (one 64-bit mask word per query and 64 nodes)
 constexpr int MAX_DEPTH = 8;
-constexpr int TREE_ROWS = 64;   // row stride of the tree K/V scratch, per layer
+constexpr int TREE_ROWS = 64;   // token rows per tile: projections and attention work on tiles of 64 tree tokens; a
+                                // context holds rows = 64 * ceil(max_tree_nodes / 64) of them (the row stride of its
+                                // per-layer tree K/V scratch and of every activation buffer)
 
 // indices into the int32 state block (MEDUSA_WS_STATE)
 enum { ST_CACHE_LEN = 0, ST_ROOT = 1, ST_BEST = 2, ST_ACCEPT_LEN = 3, ST_NEXT_ROOT = 4, ST_N_EMITTED = 5,

@@ -261,8 +261,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                             waited = true;
                             for (int p = 0; p < pend_n; ++p) {
                                 uint8_t *st = tiles + p * STAGE_BYTES;
-                                tma_load_2d(st + A_BYTES, &mapX, pend_k[p], 0, &sm->full[p], pol_keep);
-                                tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], BN, &sm->full[p], pol_keep);
+                                tma_load_2d(st + A_BYTES, &mapX, pend_k[p], a.x_row_hi, &sm->full[p], pol_keep);
+                                tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], a.x_row_lo, &sm->full[p], pol_keep);
                             }
                         }
                         if (sm->failed || !mbar_wait(&sm->empty[s], ph, a.spin_limit)) {
@@ -276,8 +276,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     mbar_expect_tx(&sm->full[s], STAGE_BYTES);
                     tma_load_2d(st, mapW, k, trow, &sm->full[s], pol_stream);
                     if (waited) {
-                        tma_load_2d(st + A_BYTES, &mapX, k, 0, &sm->full[s], pol_keep);
-                        tma_load_2d(st + A_BYTES + B_BYTES, &mapX, k, BN, &sm->full[s], pol_keep);
+                        tma_load_2d(st + A_BYTES, &mapX, k, a.x_row_hi, &sm->full[s], pol_keep);
+                        tma_load_2d(st + A_BYTES + B_BYTES, &mapX, k, a.x_row_lo, &sm->full[s], pol_keep);
                     } else {
                         pend_k[pend_n++] = k;  // n < STAGES here, so stage index == pend index
                     }
@@ -291,8 +291,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 for (int p = 0; p < pend_n; ++p) {
                     uint8_t *st = tiles + p * STAGE_BYTES;
-                    tma_load_2d(st + A_BYTES, &mapX, pend_k[p], 0, &sm->full[p], pol_keep);
-                    tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], BN, &sm->full[p], pol_keep);
+                    tma_load_2d(st + A_BYTES, &mapX, pend_k[p], a.x_row_hi, &sm->full[p], pol_keep);
+                    tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], a.x_row_lo, &sm->full[p], pol_keep);
                 }
             }
         }
@@ -446,7 +446,7 @@ bool make_tensor_map(TensorMap *out, const void *base, int rows, int K, int box_
 static_assert(sizeof(TensorMap) == sizeof(CUtensorMap), "TensorMap must mirror CUtensorMap");
 
 bool make_weight_map(TensorMap *out, const void *W, int N, int K) { return make_tensor_map(out, W, N, K, BM); }
-bool make_act_map(TensorMap *out, const void *X_planes, int K) { return make_tensor_map(out, X_planes, 2 * BN, K, BN); }
+bool make_act_map(TensorMap *out, const void *X_planes, int K, int rows) { return make_tensor_map(out, X_planes, 2 * rows, K, BN); }
 
 // CTAs resident per SM and TMA ring depth; MEDUSA_GEMM_CTAS_PER_SM / MEDUSA_GEMM_STAGES override for tuning
 static int env_int(const char *name, int dflt, int lo, int hi)
@@ -517,13 +517,15 @@ WeightPrefetch gemm_tc_prefetch_plan(const void *const *W, int n_seg, int seg_co
     p.G = pd.ctas;
     p.whole_tiles = whole_tiles ? 1 : 0;
     p.total = pd.total;
-    p.units = units;
+    // never more than a CTA's whole range (the prefetching threads walk G * units * 128 rows)
+    const long long per_cta = p.whole_tiles ? p.KB : (pd.total + p.G - 1) / p.G;
+    p.units = (long long)units < per_cta ? units : (int)per_cta;
     return p;
 }
 
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols, uint32_t spin_limit, int withhold)
+                           int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo)
 {
     if (seg0_cols <= 0) seg0_cols = seg_cols;
     static bool attr_set[64] = {};
@@ -550,6 +552,8 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     a.stages = gemm_tc_stages();
     a.spin_limit = spin_limit ? spin_limit : DEFAULT_SPIN_LIMIT;
     a.withhold = withhold;
+    a.x_row_hi = x_row_hi;
+    a.x_row_lo = x_row_lo;
     const CUtensorMap *w0 = (const CUtensorMap *)mapW[0];
     const CUtensorMap *w1 = (const CUtensorMap *)mapW[n_seg > 1 ? 1 : 0];
     const CUtensorMap *w2 = (const CUtensorMap *)mapW[n_seg > 2 ? 2 : 0];

@@ -53,6 +53,7 @@ struct GemmTcArgs {
     int stages;              // depth of the TMA ring
     uint32_t spin_limit;     // polls before a bounded wait gives up
     int withhold;            // test hook: CTA 0's producer issues no load at all, so its consumers' waits expire
+    int x_row_hi, x_row_lo;  // rows of the activation tensor where this launch's 64 token rows start in the hi / lo plane
 };
 
 // What a kernel that runs before a projection launch needs to know to pull that launch's first weight tiles into the
@@ -70,17 +71,19 @@ WeightPrefetch gemm_tc_prefetch_plan(const void *const *W, int n_seg, int seg_co
 
 // W: [N][K] bf16 row-major
 bool make_weight_map(TensorMap *out, const void *W, int N, int K);
-// X_planes: split activation, [2][64][K] bf16
-bool make_act_map(TensorMap *out, const void *X_planes, int K);
+// X_planes: split activation, [2][rows][K] bf16 (hi plane, then lo plane; rows a multiple of 64)
+bool make_act_map(TensorMap *out, const void *X_planes, int K, int rows = 64);
 int gemm_tc_num_ctas();
 int gemm_tc_stages();
 int gemm_tc_ctas_per_sm();
 // plan of a launch over n_seg weight matrices of seg_cols rows (seg_cols % 128 == 0 unless n_seg == 1); the first
 // matrix has seg0_cols rows if that is given (> 0, a multiple of 128)
 PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols = 0);
-// P[piece][t][first column of segment seg + n] = partial sums over k of (X_hi + X_lo)[t][k] * W_seg[n][k], t in [row0, T)
+// P[piece][t][first column of segment seg + n] = partial sums over k of (X_hi + X_lo)[t][k] * W_seg[n][k], t in [row0, T);
+// the launch's token rows t = 0..63 are rows x_row_hi + t and x_row_lo + t of the activation tensor (a tree of more
+// than 64 tokens is projected in tiles of 64 rows, one launch each, with P advanced by 64 rows)
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0);
+                           int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0, int x_row_hi = 0, int x_row_lo = 64);
 
 }  // namespace medusa

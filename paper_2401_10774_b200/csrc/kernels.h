@@ -45,16 +45,18 @@ void launch_silu_mul(int dtype, const float *gate_up, const PlaneDesc &pd, void 
 void launch_stream_read(const void *buf, long long bytes, float *sink, int blocks, cudaStream_t s);
 
 // ---- attention.cu ----
-// q,out: [T][H][D], k_new,v_new: [T][Hkv][D] (already rotated); caches [Hkv][L_max][D]; mask [T]; lse nullable [T][H];
+// q,out: [T][H][D], k_new,v_new: [T][Hkv][D] (already rotated); caches [Hkv][L_max][D]; mask [T][mask_words] (bit j of
+// row i: tree node j visible to query i; one word per 64 nodes); lse nullable [T][H];
 // out_lo (nullable): second plane of the split output.  Hkv divides H: query head h reads key/value head h / (H / Hkv)
 // (grouped-query attention; Hkv == H is ordinary multi-head attention).
 void launch_tree_attention_simt(int dtype, const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                 const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
-                                void *out_lo, float *lse, int T, int H, int Hkv, int D, int L_max, cudaStream_t s);
+                                void *out_lo, float *lse, int T, int H, int Hkv, int D, int L_max, cudaStream_t s,
+                                int mask_words = 1);
 
 // ---- attention_flash.cu (bf16, head_dim 128: tensor-core split-KV flash-decode kernel) ----
 constexpr int FLASH_MAX_SPLITS = 32;
-size_t tree_attention_flash_workspace_bytes(int H);
+size_t tree_attention_flash_workspace_bytes(int H, int q_tiles = 1);  // q_tiles: tiles of 64 query rows (trees > 64 nodes)
 // same contract as the kernel above; L_hint: host-side upper bound of *cache_len (the tcgen05 kernel sizes its grid
 // with it; the mma.sync kernel picks its key ranges from *cache_len on the device);
 // workspace: tree_attention_flash_workspace_bytes(H) bytes, zero-initialised once
@@ -63,7 +65,7 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
                                         int L_hint, cudaStream_t s, const void *q_lo = nullptr,
-                                        const WeightPrefetch *prefetch = nullptr);
+                                        const WeightPrefetch *prefetch = nullptr, int mask_words = 1);
 // The same operation and workspace on the tcgen05 tensor cores (attention_tc.cu): scores and P V accumulate in
 // TMEM, softmax threads own one query row each.  status: device status word (MEDUSA_ERR_TIMEOUT on an expired wait).
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,
@@ -107,7 +109,8 @@ struct PosteriorArgs {
 void launch_evaluate_posterior(const PosteriorArgs &a, cudaStream_t s);
 
 struct CommitArgs {
-    const void *tree_k, *tree_v;  // [N_L][TREE_ROWS][H][D]
+    const void *tree_k, *tree_v;  // [N_L][tree_rows][H][D]
+    int tree_rows;                // row stride of the scratch per layer (the context's rows, 64 unless it holds larger trees)
     void *k_cache, *v_cache;      // [N_L][H][L_max][D]
     const int32_t *acc_nodes, *accept_len;
     int max_commit;

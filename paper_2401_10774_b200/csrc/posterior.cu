@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(256) commit_rows_kernel(CommitArgs a)
         return;
     constexpr int VN = Vec16<AT>::N;
     const int l = blockIdx.x;
-    const AT *src = (const AT *)(blockIdx.y == 0 ? a.tree_k : a.tree_v) + (size_t)l * TREE_ROWS * a.H * a.D;
+    const AT *src = (const AT *)(blockIdx.y == 0 ? a.tree_k : a.tree_v) + (size_t)l * a.tree_rows * a.H * a.D;
     AT *dst = (AT *)(blockIdx.y == 0 ? a.k_cache : a.v_cache) + (size_t)l * a.H * a.L_max * a.D;
     const int cpr = a.D / VN;  // 16-byte chunks per head row
     const int per_node = a.H * cpr;

@@ -215,7 +215,7 @@ gemm_simt_kernel(const WT *__restrict__ X, const WT *__restrict__ Xlo, int ldx, 
                  void *__restrict__ Yv, int ldy, int col0, int T, int N, int K)
 {
     pdl_enter();
-    __shared__ float Xs[MAX_T][GS_KC + 1];
+    __shared__ float Xs[TREE_ROWS][GS_KC + 1];
     __shared__ float Ws[GS_BN][GS_KC + 1];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int n0 = blockIdx.x * GS_BN;
@@ -224,7 +224,7 @@ gemm_simt_kernel(const WT *__restrict__ X, const WT *__restrict__ Xlo, int ldx, 
     for (int r = 0; r < 8; ++r)
         acc[r][0] = acc[r][1] = 0.f;
     for (int k0 = 0; k0 < K; k0 += GS_KC) {
-        for (int i = threadIdx.x; i < MAX_T * GS_KC; i += 256) {
+        for (int i = threadIdx.x; i < TREE_ROWS * GS_KC; i += 256) {
             int r = i / GS_KC, c = i % GS_KC;
             float v = 0.f;
             if (r < T && k0 + c < K) {
@@ -284,10 +284,16 @@ static void gemm_simt_dispatch(const void *X, const void *Xlo, int ldx, const vo
 void launch_gemm_simt(int dtype, const void *X, const void *Xlo, int ldx, const void *W, void *Y, int ldy, int col0,
                       int T, int N, int K, GemmOut mode, cudaStream_t s)
 {
-    if (dtype == MEDUSA_BF16)
-        gemm_simt_dispatch<bf16>(X, Xlo, ldx, W, Y, ldy, col0, T, N, K, mode, s);
-    else
-        gemm_simt_dispatch<float>(X, nullptr, ldx, W, Y, ldy, col0, T, N, K, mode, s);
+    // the kernel covers 64 token rows: more rows run as one launch per tile of 64
+    for (int r0 = 0; r0 < T; r0 += TREE_ROWS) {
+        const int Tt = T - r0 < TREE_ROWS ? T - r0 : TREE_ROWS;
+        if (dtype == MEDUSA_BF16)
+            gemm_simt_dispatch<bf16>((const bf16 *)X + (size_t)r0 * ldx, Xlo ? (const bf16 *)Xlo + (size_t)r0 * ldx : nullptr, ldx, W,
+                                     (float *)Y + (size_t)r0 * ldy, ldy, col0, Tt, N, K, mode, s);
+        else
+            gemm_simt_dispatch<float>((const float *)X + (size_t)r0 * ldx, nullptr, ldx, W, (float *)Y + (size_t)r0 * ldy, ldy, col0,
+                                      Tt, N, K, mode, s);
+    }
 }
 
 // ---------------------------------------------------------------------------------------- rotary embedding

@@ -142,7 +142,9 @@ int32_t build_tree(const int32_t *paths, int32_t n_paths, int32_t max_depth, Tre
             return MEDUSA_ERR_INVALID_ARG;  // duplicate
     tr = TreeHost{};
     tr.T = T;
-    tr.mask.assign(T, 0);
+    const int MW = (T + 63) / 64;
+    tr.mask_words = MW;
+    tr.mask.assign((size_t)T * MW, 0);
     tr.pos.assign(T, 0);
     tr.tree_idx.assign(T, 0);
     tr.parent.assign(T, -1);
@@ -160,7 +162,9 @@ int32_t build_tree(const int32_t *paths, int32_t n_paths, int32_t max_depth, Tre
             return MEDUSA_ERR_INVALID_ARG;  // not prefix-closed
         int pi = (int)(it - nodes.begin());
         tr.parent[i] = pi;
-        tr.mask[i] = tr.mask[pi] | (1ull << i);
+        for (int w = 0; w < MW; ++w)
+            tr.mask[(size_t)i * MW + w] = tr.mask[(size_t)pi * MW + w];
+        tr.mask[(size_t)i * MW + (i >> 6)] |= 1ull << (i & 63);
         tr.pos[i] = (int32_t)t.size();
         tr.tree_idx[i] = 1 + ((int32_t)t.size() - 1) * tr.topk + t.back();
     }

@@ -3,14 +3,15 @@
 #include <cstdint>
 #include <vector>
 
-#define MEDUSA_MAX_T 64
+#define MEDUSA_MAX_T 256
 #define MEDUSA_MAX_DEPTH 8
 
 namespace medusa {
 
 struct TreeHost {
     int T = 0, P = 0, depth = 0, topk = 0;
-    std::vector<uint64_t> mask;
+    std::vector<uint64_t> mask;  // [T][mask_words]: bit j of row i (word j / 64, bit j % 64) -- node j is i or an ancestor
+    int mask_words = 1;          // ceil(T / 64)
     std::vector<int32_t> pos, tree_idx, parent, retrieve;  // retrieve: [P][depth+1]
 };
 

@@ -41,6 +41,14 @@ TREE_SPECS = {
     "sparse64_d4": dict(per_depth_topk=(4, 3, 2, 2), n_nodes=64),
     "sparse64_d5": dict(per_depth_topk=(4, 3, 2, 2, 2), n_nodes=64),
 }
+# Trees of more than 64 nodes (the paper's Sec. 3.3.1 / Fig. 4 studies sparse trees of up to 256 nodes): the same
+# surrogate construction (score prod 1/(rank+1), best n nodes), wider per-depth top-k.
+LARGE_TREE_SPECS = {
+    "sparse128_d4": dict(per_depth_topk=(6, 4, 3, 2), n_nodes=128),
+    "sparse256_d4": dict(per_depth_topk=(10, 6, 4, 3), n_nodes=256),
+    "sparse256_d5": dict(per_depth_topk=(10, 6, 4, 3, 2), n_nodes=256),
+    "sparse100_d3": dict(per_depth_topk=(7, 5, 3), n_nodes=100),
+}
 
 
 def model_shape(name: str, **override) -> dict:

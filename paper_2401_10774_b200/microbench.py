@@ -36,6 +36,9 @@ def main():
     ap.add_argument("--attention", type=int, default=0, metavar="L", help="time tree_attention alone at cache length L")
     ap.add_argument("--caches", type=int, default=32)
     ap.add_argument("--weight-prefetch", type=int, default=None, metavar="TILES")
+    ap.add_argument("--device-weights", action="store_true",
+                    help="draw the weights on the device (N(0, 0.02^2), not the seeded host recipe): seconds instead of a "
+                         "minute of set-up, for timing runs whose numbers do not depend on the values")
     args = ap.parse_args()
     if args.attention:
         return attention_only(args)
@@ -43,13 +46,28 @@ def main():
     cfg = I.model_shape(args.model, n_layers=args.layers)
     tree_name = args.tree or ("sparse64_d5" if cfg["n_medusa"] >= 5 else "sparse64_d4")
     spec = I.TREE_SPECS[tree_name]
-    w = I.make_weights(cfg, seed=40, dtype="bf16")
+    if args.device_weights:
+        gen = torch.Generator(device="cuda").manual_seed(40)
 
-    def dev(a):
-        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda().view(torch.bfloat16)
+        def rnd(*shape, std=0.02, mean=0.0):
+            return (torch.randn(*shape, device="cuda", generator=gen) * std + mean).bfloat16()
 
-    dw = {k: dev(v) for k, v in w.items() if k != "layers"}
-    dw["layers"] = [{k: dev(v) for k, v in lw.items()} for lw in w["layers"]]
+        d, F, V, K = cfg["d"], cfg["ffn"], cfg["vocab"], cfg["n_medusa"]
+        hd, hkd = cfg["n_heads"] * cfg["head_dim"], I.kv_heads(cfg) * cfg["head_dim"]
+        dw = dict(embed=rnd(V, d), lm_head=rnd(V, d), final_norm=rnd(d, std=0.0, mean=1.0), medusa_w1=rnd(K, d, d),
+                  medusa_w2=rnd(K, V, d), layers=[])
+        for _ in range(cfg["n_layers"]):
+            dw["layers"].append(dict(attn_norm=rnd(d, std=0.0, mean=1.0), wq=rnd(hd, d), wk=rnd(hkd, d), wv=rnd(hkd, d),
+                                     wo=rnd(d, hd), ffn_norm=rnd(d, std=0.0, mean=1.0), w_gate=rnd(F, d), w_up=rnd(F, d),
+                                     w_down=rnd(d, F)))
+    else:
+        w = I.make_weights(cfg, seed=40, dtype="bf16")
+
+        def dev(a):
+            return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda().view(torch.bfloat16)
+
+        dw = {k: dev(v) for k, v in w.items() if k != "layers"}
+        dw["layers"] = [{k: dev(v) for k, v in lw.items()} for lw in w["layers"]]
     ctx = B.Context(cfg, B.BF16, args.L_max)
     ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
     if args.weight_prefetch is not None:

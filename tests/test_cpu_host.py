@@ -77,13 +77,26 @@ def test_host_tree_buffers_bit_exact_vs_oracle(oracle, name):
             assert np.array_equal(t_lib[k], t_ora[k]), k
 
 
+@pytest.mark.parametrize("topk,n_nodes", [((6, 4, 3, 2, 2), 128), ((10, 6, 4, 3, 2), 256)])
+def test_host_large_tree_buffers_bit_exact_vs_oracle(oracle, topk, n_nodes):
+    # trees of more than 64 nodes (Sec. 3.3.1, Fig. 4): masks of several 64-bit words per node
+    p_lib, p_ora = B.default_tree_paths(topk, n_nodes), oracle.default_tree_paths(topk, n_nodes)
+    assert {tuple(r) for r in p_lib.tolist()} == {tuple(r) for r in p_ora.tolist()}
+    t_lib, t_ora = B.build_tree_buffers(None, p_lib), oracle.build_tree_buffers(p_ora[::-1])
+    assert t_lib["mask"].shape == (n_nodes, (n_nodes + 63) // 64)
+    for k in ("T", "P", "depth", "topk"):
+        assert t_lib[k] == t_ora[k]
+    for k in ("mask", "pos", "tree_idx", "parent", "retrieve"):
+        assert np.array_equal(t_lib[k], t_ora[k]), k
+
+
 def test_host_tree_random_prefix_closed_trees(oracle):
     g = I.rng(17, "random-trees")
     for trial in range(40):
         depth = int(g.integers(1, 6))
         nodes = {()}
-        target = int(g.integers(1, 64))
-        for _ in range(2000):
+        target = int(g.integers(1, 64)) if trial % 3 else int(g.integers(65, 257))  # a third of them: multi-word masks
+        for _ in range(8000):
             if len(nodes) >= target:
                 break
             par = sorted(nodes)[int(g.integers(0, len(nodes)))]
@@ -115,7 +128,7 @@ def test_tree_from_accuracies_bit_exact_vs_oracle(oracle):
         if trial % 3 == 2:
             g.shuffle(acc, axis=1)           # rows need not be sorted by rank
         total = sum(topk ** k for k in range(1, depth + 1))
-        cases.append((np.ascontiguousarray(acc), int(min(64, 1 + total, g.integers(2, 65)))))
+        cases.append((np.ascontiguousarray(acc), int(min(256, 1 + total, g.integers(2, 257 if len(cases) % 2 else 65)))))
     cases.append((np.array([[1 / (i + 1) for i in range(10)]] * 4), 64))
     for acc, n_nodes in cases:
         p_lib, e_lib = B.tree_paths_from_accuracies(acc, n_nodes)
@@ -133,7 +146,7 @@ def test_tree_from_accuracies_bit_exact_vs_oracle(oracle):
     d = B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"])
     assert {tuple(r) for r in p.tolist()} == {tuple(r) for r in d.tolist()}
     for bad, n in ((np.array([[1.5]]), 2), (np.array([[float("nan")]]), 2), (np.array([[0.5, 0.1]]), 4),
-                   (np.full((2, 16), 0.5), 66)):
+                   (np.full((2, 16), 0.5), 258)):
         with pytest.raises(B.MedusaError) as e:
             B.tree_paths_from_accuracies(bad, n)
         assert e.value.code in (B.ERR_INVALID_ARG, B.ERR_SHAPE)
@@ -145,7 +158,7 @@ def test_host_tree_rejects_invalid_input():
         with pytest.raises(B.MedusaError) as e:
             B.build_tree_buffers(None, p.astype(np.int32))
         assert e.value.code == B.ERR_INVALID_ARG
-    too_many = np.array([[i] for i in range(64)], dtype=np.int32)  # 65 nodes
+    too_many = np.array([[i] for i in range(256)], dtype=np.int32)  # 257 nodes
     with pytest.raises(B.MedusaError) as e:
         B.build_tree_buffers(None, too_many)
     assert e.value.code == B.ERR_SHAPE
