@@ -31,7 +31,8 @@ from paper_2401_10774_b200 import roofline as R  # noqa: E402
 # The default (and the headline) is the 7B greedy step; `--workload 13b` measures the 13B-shape step with five
 # heads, the depth-5 tree, typical acceptance with a Gumbel-sampled root and a 3584-token prompt; `--workload 7b_long`
 # is the 7B step against a nearly full cache (3840-token prompt, capacity 4096); `--workload mistral7b` is the shape of
-# the paper's Zephyr-7B backbone (grouped-query attention, 8 key/value heads) with five heads and typical acceptance.
+# the paper's Zephyr-7B backbone (grouped-query attention, 8 key/value heads) with five heads and typical acceptance;
+# `--workload 7b_tree128 / 7b_tree256` are the 7B step with larger trees.
 WORKLOADS = {
     "7b": dict(name="7b_medusa1_greedy_step", model="7b", tree="sparse64_d4", prompt=512, L_max=4096, weights_seed=40,
                prompt_seed=41, mode="greedy", oracle_layers=8,
@@ -45,12 +46,24 @@ WORKLOADS = {
                       oracle_layers=4,
                       metric="decode tokens/s (Mistral-7B-shape bf16 Medusa tree-verification step, grouped-query attention "
                              "with 8 key/value heads, 5 heads, 64-node depth-5 tree, typical acceptance, batch 1)"),
+    # trees of more than 64 nodes (the paper's Fig. 4 studies up to 256): the same 7B step with the 128- / 256-node
+    # surrogate trees; the token rows are processed in tiles of 64, the weights streamed once per tile
+    "7b_tree128": dict(name="7b_medusa1_greedy_step_tree128", model="7b", tree="sparse128_d4", prompt=512, L_max=4096,
+                       weights_seed=40, prompt_seed=41, mode="greedy", oracle_layers=2,
+                       metric="decode tokens/s (7B-shape bf16 Medusa tree-verification step, 128-node tree, batch 1)"),
+    "7b_tree256": dict(name="7b_medusa1_greedy_step_tree256", model="7b", tree="sparse256_d4", prompt=512, L_max=4096,
+                       weights_seed=40, prompt_seed=41, mode="greedy", oracle_layers=1,
+                       metric="decode tokens/s (7B-shape bf16 Medusa tree-verification step, 256-node tree, batch 1)"),
     "13b": dict(name="13b_medusa_typical_step", model="13b", tree="sparse64_d5", prompt=3584, L_max=4096, weights_seed=50,
                 prompt_seed=51, noise_seed=52, mode="typical", temperature=0.7, eps=0.09, delta=0.3, oracle_layers=4,
                 metric="decode tokens/s (13B-shape bf16 Medusa tree-verification step, 64-node depth-5 tree, typical "
                        "acceptance, batch 1)"),
 }
 WORKLOAD = WORKLOADS["7b"]
+
+
+def tree_spec(name: str) -> dict:
+    return I.LARGE_TREE_SPECS[name] if name in I.LARGE_TREE_SPECS else I.TREE_SPECS[name]
 
 
 def measured_peaks():
@@ -134,7 +147,7 @@ class OracleSample:
         self.n = n_sample_layers
         self.cfg_full = cfg_full
         self.L = L
-        spec = I.TREE_SPECS[WORKLOAD["tree"]]
+        spec = tree_spec(WORKLOAD["tree"])
         self.tree = O.build_tree_buffers(O.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
         cfg = dict(cfg_full, n_layers=n_sample_layers)
         self.w = I.make_weights(cfg, seed=WORKLOAD["weights_seed"], dtype="bf16")
@@ -196,7 +209,7 @@ def run_reference(args):
         # each timed step runs 1 of the identical decoder layers; ms_per_step is that sample scaled to the full depth,
         # so steps x ms_per_step exceeds the wall time of this run by design
         "extrapolated": True, "layers_run_per_step": 1, "layers_total": cfg["n_layers"],
-        "config": {"workload": WORKLOAD["name"], "tree_nodes": 64, "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"]},
+        "config": {"workload": WORKLOAD["name"], "tree_nodes": tree_spec(WORKLOAD["tree"])["n_nodes"], "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"]},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -246,8 +259,8 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    cfg = I.model_shape(WORKLOAD["model"])
-    spec = I.TREE_SPECS[WORKLOAD["tree"]]
+    spec = tree_spec(WORKLOAD["tree"])
+    cfg = I.model_shape(WORKLOAD["model"], max_tree_nodes=spec["n_nodes"])
     t_setup = time.perf_counter()
     w = I.make_weights(cfg, seed=WORKLOAD["weights_seed"], dtype="bf16")
 
@@ -263,8 +276,6 @@ def run_gpu(args):
     torch.cuda.set_stream(stream)
     ctx = B.Context(cfg, B.BF16, WORKLOAD["L_max"], device=local, stream=stream.cuda_stream)
     tree = ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
-    if args.weight_prefetch is not None:
-        ctx.set_option(B.OPT_WEIGHT_PREFETCH, args.weight_prefetch)
     ctx.load_weights(dw)
     prompt = I.make_prompt(WORKLOAD["prompt"], cfg["vocab"], WORKLOAD["prompt_seed"])
     ctx.prefill(torch.from_numpy(prompt).cuda())
@@ -407,7 +418,6 @@ def run_gpu(args):
             "data": "synthetic",
             "config": {"workload": WORKLOAD["name"], "tree_nodes": T, "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"],
                        "cache_len_start": L0, "heads": cfg["n_medusa"], "replicas": world,
-                       "weight_prefetch_tiles": "library default" if args.weight_prefetch is None else args.weight_prefetch,
                        "l2": "inputs larger than L2: every step streams %.1f GB of weights" % (sb["gemm_weights"] / 1e9)},
             "clocks": clocks,
             "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": "tokens/s",
@@ -467,9 +477,6 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS), help="7b: the headline configuration")
-    ap.add_argument("--weight-prefetch", type=int, default=None, metavar="TILES",
-                    help="comparison runs: weight tiles per projection CTA that the in-between kernels pull into the L2 "
-                         "(library default if not given, 0 = off)")
     args = ap.parse_args()
     global WORKLOAD
     WORKLOAD = WORKLOADS[args.workload]

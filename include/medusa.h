@@ -127,13 +127,10 @@ enum {
                                       * buffers (parity checks layer by layer); -1 (default) off */
     MEDUSA_OPT_SPIN_LIMIT = 4,       /* polls after which a bounded device-side wait gives up with MEDUSA_ERR_TIMEOUT;
                                       * 0 = the kernels' default (about 4 million) */
-    MEDUSA_OPT_WITHHOLD_LOAD = 5,    /* failure-path test hook, one shot: 1 = in the next tensor-core GEMM launch, 2 = in the
+    MEDUSA_OPT_WITHHOLD_LOAD = 5     /* failure-path test hook, one shot: 1 = in the next tensor-core GEMM launch, 2 = in the
                                       * next tcgen05 attention launch, one CTA's producer issues no load at all, so that its
                                       * consumers' bounded waits expire with nothing in flight; the launch returns, its output
                                       * is unusable and the device status becomes MEDUSA_ERR_TIMEOUT */
-    MEDUSA_OPT_WEIGHT_PREFETCH = 6   /* weight tiles (128 rows x 64 columns) per projection CTA that the kernel running in
-                                      * front of a projection pulls into the L2 while the HBM would otherwise idle;
-                                      * default 8, 0 = off.  Never changes a result. */
 };
 
 /* ---- lifetime ------------------------------------------------------------------------------------ */

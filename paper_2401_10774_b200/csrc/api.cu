@@ -60,9 +60,6 @@ struct medusa_ctx {
     void *tap_att = nullptr;                          // the layer's attention output as the o projection reads it
     void *tap_xn_out = nullptr;                       // normalised residual stream after the layer (next norm's gain)
     // test hooks for the bounded device-side waits (MEDUSA_OPT_SPIN_LIMIT, MEDUSA_OPT_WITHHOLD_LOAD)
-    // (tile, k block) pairs per projection CTA that the kernel in front of a projection pulls into the L2 (prefetch.cuh);
-    // 0 = off (MEDUSA_OPT_WEIGHT_PREFETCH)
-    int prefetch_units = 0;
     uint32_t spin_limit = 0;  // 0: the kernels' default
     int withhold = 0;         // one-shot: 1 = next tensor-core GEMM launch, 2 = next tcgen05 attention launch
     // host-side upper bound of the device-resident cache length (a hint for attention kernels that size their
@@ -226,7 +223,7 @@ struct ProfScope {
 // Tree attention of one layer: tensor-core flash kernel for bf16 / head_dim 128, CUDA-core kernel otherwise.
 int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v_new, const void *kc, const void *vc,
                   const int32_t *cache_len, const uint64_t *mask, void *out, void *out_lo, float *lse, int T, int L_hint,
-                  bool in_step, int mask_words, const void *q_lo = nullptr, const WeightPrefetch *pf = nullptr)
+                  bool in_step, int mask_words, const void *q_lo = nullptr)
 {
     const medusa_model_desc &m = c->m;
     if (c->flash_ws) {
@@ -245,7 +242,7 @@ int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v
         }
         else
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_flash(q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse,
-                                                                     c->flash_ws, T, m.n_heads, c->Hkv, m.L_max, L_hint, c->stream, q_lo, pf, mask_words));
+                                                                     c->flash_ws, T, m.n_heads, c->Hkv, m.L_max, L_hint, c->stream, q_lo, mask_words));
         if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "flash attention launch failed: %s", cudaGetErrorString(e));
         return MEDUSA_OK;
     }
@@ -266,18 +263,20 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
     if (seg0_cols <= 0) seg0_cols = seg_cols;
     if (c->use_tc && (n_seg == 1 || (seg_cols % 128 == 0 && seg0_cols % 128 == 0))) {
         const TensorMap *maps[3] = {mapW, mapW + (n_seg > 1 ? 1 : 0), mapW + (n_seg > 2 ? 2 : 0)};
-        *pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, (long long)plane_stride, seg0_cols);
+        // up to 64 rows: one launch of one token tile; more: launches of two token tiles (128 rows) each, so that the
+        // weights are streamed once per 128 rows
+        const int RT = gemm_tc_row_tiles(T), rows_per_launch = RT * TREE_ROWS;
+        *pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, (long long)plane_stride, seg0_cols, RT);
         if (!whole_tiles && (size_t)pd->n_max * plane_stride > c->part_elems)
             return fail(c, MEDUSA_ERR_SHAPE, "projection needs %d partial planes, more than the workspace holds", pd->n_max);
-        // the kernel covers 64 token rows: a larger tree is projected tile by tile (one launch per 64 rows, the weights
-        // streamed once per tile), every tile with the same plan, so the consumer finds the same pieces in every row
-        for (int r0 = (row0 / TREE_ROWS) * TREE_ROWS; r0 < T; r0 += TREE_ROWS) {
+        // every launch of the projection uses the same plan, so the consumer finds the same pieces in every row
+        for (int r0 = (row0 / rows_per_launch) * rows_per_launch; r0 < T; r0 += rows_per_launch) {
             cudaError_t e = cudaSuccess;
             const int wh = c->withhold == 1 ? 1 : 0;
             if (wh) c->withhold = 0;
-            const int Tt = T - r0 < TREE_ROWS ? T - r0 : TREE_ROWS, row0t = row0 > r0 ? row0 - r0 : 0;
+            const int Tt = T - r0 < rows_per_launch ? T - r0 : rows_per_launch, row0t = row0 > r0 ? row0 - r0 : 0;
             PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, n_seg, seg_cols, K, *pd, P + (size_t)r0 * ldy, ldy, Tt, row0t,
-                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0));
+                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0, RT));
             if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "tensor-core GEMM launch failed: %s", cudaGetErrorString(e));
         }
         return MEDUSA_OK;
@@ -309,17 +308,8 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
     PROF(c, PC_ELEMWISE, 1, launch_rope_table(c->rope_cs, cache_len, pos, T, D, m.rope_theta, s));
     MEDUSA_LAUNCH_CHECK(c);
     PlaneDesc pd_prev{};  // planes of the previous projection still to be added to the residual stream
-    // weight prefetch by the kernels between the projections: only where the tensor-core projection follows
-    const int pfu = c->use_tc && HD % 128 == 0 && HkvD % 128 == 0 && F % 128 == 0 && d % 128 == 0 ? c->prefetch_units : 0;
     for (int l = 0; l < m.n_layers; ++l) {
         const void *const *w = c->layers.data() + (size_t)l * 9;
-        const void *w_o[3] = {w[4], w[4], w[4]}, *w_gu[3] = {w[6], w[7], w[7]}, *w_dn[3] = {w[8], w[8], w[8]};
-        const void *w_qkv[3] = {w[1], w[2], w[3]};
-        const WeightPrefetch pf_qkv = gemm_tc_prefetch_plan(w_qkv, 3, HkvD, d, false, HD, pfu);
-        // the attention kernel and the rotation in front of it leave the HBM idle for long: the whole output projection
-        const WeightPrefetch pf_o = gemm_tc_prefetch_plan(w_o, 1, d, HD, false, d, pfu ? 1 << 20 : 0);
-        const WeightPrefetch pf_gu = gemm_tc_prefetch_plan(w_gu, 2, F, d, false, F, pfu);
-        const WeightPrefetch pf_dn = gemm_tc_prefetch_plan(w_dn, 1, d, F, false, d, pfu);
         const TensorMap *wm = c->use_tc ? c->wmaps.data() + (size_t)l * 7 : nullptr;
         char *tk = (char *)c->tree_k + (size_t)l * c->rows * HkvD * c->esz;
         char *tv = (char *)c->tree_v + (size_t)l * c->rows * HkvD * c->esz;
@@ -328,7 +318,7 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
         PlaneDesc pd{};
         // x += down-projection of the previous layer;  xn = RMSNorm(x)
         PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd_prev, w[0], m.rms_eps, c->xn, c->lo(c->xn, d), nullptr, T,
-                                                   d, s, &pf_qkv));
+                                                   d, s));
         if (c->tap_layer >= 0) {
             const size_t planes = dt == MEDUSA_BF16 ? 2 : 1;
             if (l == c->tap_layer)
@@ -354,26 +344,23 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
         }
         MEDUSA_LAUNCH_CHECK(c);
         TRY(attention(c, c->q, tk, tv, kc, vc, cache_len, mask, c->att, c->lo(c->att, HD), nullptr, T, c->L_upper, true,
-                      mask_words, c->lo(c->q, HD), &pf_o));
+                      mask_words, c->lo(c->q, HD)));
         if (l == c->tap_layer)
             MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_att, c->att, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)c->rows * HD * c->esz,
                                            cudaMemcpyDeviceToDevice, s));
         const void *wo[1] = {w[4]};
         TRY(project(c, c->att, &c->map_att, wo, wm ? wm + 3 : nullptr, 1, d, HD, c->part, (size_t)c->rows * d, d, T, 0, false, &pd));
         // x += attention output projection;  xn = RMSNorm(x)
-        PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd, w[5], m.rms_eps, c->xn, c->lo(c->xn, d), nullptr, T, d, s,
-                                                   &pf_gu));
+        PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd, w[5], m.rms_eps, c->xn, c->lo(c->xn, d), nullptr, T, d, s));
         const void *wgu[2] = {w[6], w[7]};
         TRY(project(c, c->xn, &c->map_xn, wgu, wm ? wm + 4 : nullptr, 2, F, d, c->part, (size_t)c->rows * 2 * F, 2 * F, T, 0, false, &pd));
-        PROF(c, PC_ELEMWISE, 1, launch_silu_mul(dt, c->part, pd, c->act, c->lo(c->act, F), T, F, s, &pf_dn));
+        PROF(c, PC_ELEMWISE, 1, launch_silu_mul(dt, c->part, pd, c->act, c->lo(c->act, F), T, F, s));
         MEDUSA_LAUNCH_CHECK(c);
         const void *wd[1] = {w[8]};
         TRY(project(c, c->act, &c->map_act, wd, wm ? wm + 6 : nullptr, 1, d, F, c->part, (size_t)c->rows * d, d, T, 0, false, &pd_prev));
     }
-    const void *w_lm[3] = {c->w.lm_head, c->w.lm_head, c->w.lm_head};
-    const WeightPrefetch pf_lm = gemm_tc_prefetch_plan(w_lm, 1, m.vocab, d, true, m.vocab, c->use_tc && d % 128 == 0 ? c->prefetch_units : 0);
     PROF(c, PC_ELEMWISE, 1, launch_add_rmsnorm(dt, c->x, c->part, pd_prev, c->w.final_norm, m.rms_eps, c->hidden,
-                                               c->lo(c->hidden, d), c->hidden_f32, T, d, s, &pf_lm));
+                                               c->lo(c->hidden, d), c->hidden_f32, T, d, s));
     if (c->tap_layer >= 0 && c->tap_layer == m.n_layers - 1) {
         MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_x_out, c->x, (size_t)c->rows * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
         MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_xn_out, c->hidden, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)c->rows * d * c->esz,
@@ -634,13 +621,6 @@ extern "C" int32_t medusa_set_option(medusa_ctx *c, int32_t option, int64_t valu
         MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
         drop_step_graphs(c);  // captured launches carry the old limit
         c->spin_limit = (uint32_t)value;
-        return MEDUSA_OK;
-    case MEDUSA_OPT_WEIGHT_PREFETCH:
-        if (value < 0 || value > 1024) return fail(c, MEDUSA_ERR_INVALID_ARG, "weight prefetch: 0 (off) to 1024 tiles per projection CTA");
-        MEDUSA_CUDA(c, cudaSetDevice(c->device));
-        MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
-        drop_step_graphs(c);
-        c->prefetch_units = (int)value;
         return MEDUSA_OK;
     case MEDUSA_OPT_WITHHOLD_LOAD:
         if (value < 0 || value > 2) return fail(c, MEDUSA_ERR_INVALID_ARG, "withhold: 0 (off), 1 (next tensor-core GEMM) or 2 (next tcgen05 attention)");

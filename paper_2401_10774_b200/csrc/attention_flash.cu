@@ -19,7 +19,6 @@
 #include "common.cuh"
 #include "pdl.cuh"
 #include "kernels.h"
-#include "prefetch.cuh"
 
 namespace medusa {
 
@@ -32,8 +31,8 @@ constexpr int STAGES = 3;
 constexpr int THREADS = 256;     // 8 warps: warp w owns query rows 16*(w&3).. and key half (w>>2) of every tile
 constexpr int TILE_BYTES = BKEY * D * 2;           // 16 KiB for K, same for V
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
-constexpr int Q_BYTES = 2 * TILE_BYTES;                         // Q tile and its second plane (zeros without one)
-constexpr int SMEM_BYTES = Q_BYTES + STAGES * STAGE_BYTES;      // Q planes, then the K/V ring
+// Q tile (and its second plane, if q comes as two planes), then the K/V ring
+constexpr int smem_bytes(bool qlo) { return (qlo ? 2 : 1) * TILE_BYTES + STAGES * STAGE_BYTES; }
 constexpr float LOG2E = 1.4426950408889634f;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -73,21 +72,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 struct Args {
     const bf16 *q, *k_new, *v_new;   // [T][H][D]
-    const bf16 *q_lo;                // nullable [T][H][D]: second plane of q (scores are q.k + q_lo.k)
+    const bf16 *q_lo;                // [T][H][D] second plane of q (kernels instantiated with QLO): scores are q.k + q_lo.k
     const bf16 *k_cache, *v_cache;   // [H][L_max][D]
     const int32_t *cache_len;
     const uint64_t *mask;            // [T][mask_words]: bit j of row i -- tree node j visible to query i
-    int mask_words;                  // 64 tree nodes per word
-    int q_tiles;                     // tiles of 64 query rows (gridDim.z); a query tile sees the tree's key tiles 0..its own
+    int mask_words;                  // 64 tree nodes per word (1 unless the kernel is instantiated with LARGE)
     bf16 *out, *out_lo;              // [T][H][D]; out_lo nullable
     float *lse;                      // nullable [T][H]
-    float *ws_o;                     // [q_tiles][H][max_splits][64][128] unnormalised partial outputs
-    float *ws_ml;                    // [q_tiles][H][max_splits][2][64]  running max (log2 domain) and sum
-    int *counters;                   // [q_tiles][H] arrival tickets, zero between launches
+    float *ws_o;                     // [q tiles][H][max_splits][64][128] unnormalised partial outputs
+    float *ws_ml;                    // [q tiles][H][max_splits][2][64]  running max (log2 domain) and sum
+    int *counters;                   // [q tiles][H] arrival tickets, zero between launches
     int T, H, L_max, tiles_per_split, max_splits;
     int Hkv;                         // key/value heads; query head h reads key/value head h / (H / Hkv)
     int rows_max_tiles;              // caches of up to this many tiles run in row-split mode (0: never)
-    WeightPrefetch pf;               // weight tiles of the projection that follows, asked for before the dependency wait
 };
 
 // loads one 64-key tile pair (K and V) into a stage; rows >= n_valid are zero-filled
@@ -111,10 +108,10 @@ __device__ __forceinline__ void load_tile(uint8_t *stage, const bf16 *ksrc, cons
 // (Twice the CTAs of one key range per head at half the tensor work per tile each; K/V are read twice, the second
 // time from L2.)  Its tile loop repeats the key-range form's with 16 instead of 32 keys per warp; the two are kept
 // spelled out because one template for both measured 2-10 % slower (register allocation of the longer form).
+template <bool QLO>
 __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem_all, int h, int half, int L, int nt)
 {
-    uint8_t *smem = smem_all + Q_BYTES;
-    const bool has_qlo = a.q_lo != nullptr;
+    uint8_t *smem = smem_all + (QLO ? 2 : 1) * TILE_BYTES;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 1, kq = warp >> 1;
     const int rbase = half * 32;
@@ -140,7 +137,7 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
             const int r = idx >> 4, c = idx & 15;
             const bool ok = rbase + r < a.T;
             cp_async16(qb + tile_off(r, c), a.q + (size_t)(ok ? rbase + r : 0) * HD + (size_t)h * D + c * 8, ok);
-            if (has_qlo)
+            if (QLO)
                 cp_async16(qb + TILE_BYTES + tile_off(r, c), a.q_lo + (size_t)(ok ? rbase + r : 0) * HD + (size_t)h * D + c * 8, ok);
         }
         cp_async_commit();
@@ -154,7 +151,7 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
     __syncthreads();
     uint32_t qf[8][4];
     const int q_row = wq * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
-    const uint32_t q_lo_addr = smem_u32(smem_all) + TILE_BYTES;
+    const uint32_t q_lo_addr = smem_u32(smem_all) + TILE_BYTES;  // second plane's tile (QLO): fragments are re-read per tile
     {
         const uint32_t qb = smem_u32(smem_all);
 #pragma unroll
@@ -190,7 +187,7 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
             ldsm_x4(kb + tile_off(kr, 2 * ks + ((lane >> 3) & 1)), b0, b1, b2, b3);
             mma_bf16(s[0], qf[ks], b0, b1);
             mma_bf16(s[1], qf[ks], b2, b3);
-            if (has_qlo) {  // the second plane's fragments come from shared memory: no registers to hold them
+            if (QLO) {  // the second plane's fragments come from shared memory: there are no registers to hold them
                 uint32_t ql[4];
                 ldsm_x4(q_lo_addr + tile_off(q_row, 2 * ks + (lane >> 4)), ql[0], ql[1], ql[2], ql[3]);
                 mma_bf16(s[0], ql, b0, b1);
@@ -334,109 +331,70 @@ __device__ __forceinline__ void attention_rows_mode(const Args &a, uint8_t *smem
     }
 }
 
-// The key ranges of a launch: which form runs, how many ranges, and one CTA's tiles -- all derived from the cache length.
-struct Ranges {
-    int L, nt, n_active, tile0, tile1, n_tiles;
-    bool rows_mode, has_tree, idle;
-};
-__device__ __forceinline__ Ranges plan_ranges(const Args &a, int L_raw, int sp)
-{
-    Ranges r;
-    // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
-    r.L = min(max(L_raw, 0), a.L_max);
-    r.nt = (r.L + BKEY - 1) / BKEY;
-    r.rows_mode = r.nt <= a.rows_max_tiles && gridDim.y >= 2 && a.q_tiles == 1;
-    // Key ranges: fixed by the launch (tiles_per_split > 0), or chosen here from the true cache length, so that the
-    // result does not depend on what the host knew about the length when it launched: as many ranges as the grid has
-    // rows (one wave of CTAs; every CTA requests its first tiles before the dependency wait, so a range costs little
-    // to start), but no range shorter than two tiles.
-    int tps = a.tiles_per_split;
-    if (tps <= 0) {
-        const int want = min((int)gridDim.y, max(1, r.nt / 2));
-        tps = r.nt > 0 ? (r.nt + want - 1) / want : 1;
-    }
-    const int n_cache_splits = (r.nt + tps - 1) / tps;
-    // never more ranges than the grid has rows: when the launch's fixed range size was chosen for a shorter cache than
-    // the one found here, the last range takes all the remaining tiles (slower, still complete)
-    r.n_active = min(n_cache_splits > 0 ? n_cache_splits : 1, (int)gridDim.y);
-    r.idle = sp >= r.n_active;
-    r.tile0 = sp * tps;
-    r.has_tree = sp == r.n_active - 1;
-    r.tile1 = r.has_tree ? r.nt : min(r.nt, r.tile0 + tps);
-    // the last range also takes the tree's own keys: query tile z needs the key tiles 0..z (ancestors come first)
-    r.n_tiles = (r.tile1 - r.tile0) + (r.has_tree ? (int)blockIdx.z + 1 : 0);
-    return r;
-}
-
+// QLO: q comes as two bf16 planes (the decode step's rotation kernel writes them), and the scores are q.k + q_lo.k, so
+// that q's rounding to one plane does not reach the softmax.  LARGE: trees of more than 64 nodes -- blockIdx.z is the
+// tile of 64 query rows, which sees the tree's key tiles 0..z (ancestors have smaller indices) through one 64-bit mask
+// word per key tile.  The plain instantiation is the 64-node kernel unchanged.
+template <bool QLO, bool LARGE>
 __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a)
 {
-    pdl_trigger();
+    pdl_enter();
     extern __shared__ __align__(1024) uint8_t smem_all[];
-    uint8_t *smem = smem_all + Q_BYTES;  // K/V ring; the Q planes sit in front of it
-    const bool has_qlo = a.q_lo != nullptr;
+    uint8_t *smem = smem_all + (QLO ? 2 : 1) * TILE_BYTES;  // K/V ring; the Q tile(s) sit in front of it
     __shared__ int s_ticket;
     const int h = blockIdx.x, sp = blockIdx.y;
-    const int q0 = (int)blockIdx.z * BQ;      // first query row of this CTA's tile
-    const int Tq = min(BQ, a.T - q0);         // its query rows
+    const int q0 = LARGE ? (int)blockIdx.z * BQ : 0;            // first query row of this CTA's tile
+    const int Tq = LARGE ? min(BQ, a.T - q0) : a.T;             // its query rows
+    const int tree_tiles = LARGE ? (int)blockIdx.z + 1 : 1;     // key tiles of the tree this query tile can see
+    const size_t slot = LARGE ? (size_t)blockIdx.z * a.H + h : (size_t)h;  // (query tile, head)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 3, kh = warp >> 2;  // query-row group, key half
+    // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
+    const int L = min(max(*a.cache_len, 0), a.L_max);
+    const int nt = (L + BKEY - 1) / BKEY;
+    if (!LARGE && nt <= a.rows_max_tiles && gridDim.y >= 2) {
+        if (sp < 2)
+            attention_rows_mode<QLO>(a, smem_all, h, sp, L, nt);
+        return;
+    }
+    // Key ranges: fixed by the launch (tiles_per_split > 0), or chosen here from the true cache length, so that
+    // the result does not depend on what the host knew about the length when it launched.  A CTA's time grows
+    // with its tiles, the combine with the number of ranges: about sqrt(tiles) ranges balances the two, and never
+    // more ranges than the grid has rows.
+    int tps = a.tiles_per_split;
+    if (tps <= 0) {
+        int want = 1;
+        while (want * want < nt) ++want;
+        if (want > (int)gridDim.y) want = (int)gridDim.y;
+        tps = nt > 0 ? (nt + want - 1) / want : 1;
+    }
+    const int n_cache_splits = (nt + tps - 1) / tps;
+    // never more ranges than the grid has rows: when the launch's fixed range size was chosen for a shorter cache than
+    // the one found here, the last range takes all the remaining tiles (slower, still complete)
+    const int n_active = min(n_cache_splits > 0 ? n_cache_splits : 1, (int)gridDim.y);
+    if (sp >= n_active)
+        return;
+    const int tile0 = sp * tps;
+    const bool has_tree = sp == n_active - 1;
+    const int tile1 = has_tree ? nt : min(nt, tile0 + tps);
+    const int n_tiles = (tile1 - tile0) + (has_tree ? tree_tiles : 0);
     const size_t HD = (size_t)a.H * D, HkvD = (size_t)a.Hkv * D;
     const int hk = h / (a.H / a.Hkv);
-    // ---- before the dependency wait: request this CTA's first cache tiles.  The cache rows below the cache length, and
-    // the length itself, were written by the previous step's commit (or the prefill): kernels that had finished before
-    // the kernel in front of this one could start.  What the kernel in front writes are q and the tree's own keys and
-    // values, which are requested after the wait.  The length is read again after the wait; should it differ (never
-    // observed), the prefetched tiles are dropped and requested again.
-    Ranges rg = plan_ranges(a, *a.cache_len, sp);
-    auto prefetch_cache_tiles = [&]() {
-        if (rg.rows_mode || rg.idle)
-            return;
-        for (int i = 0; i < STAGES - 1; ++i) {
-            const int ct = rg.tile0 + i;
-            if (ct < rg.tile1) {
-                const size_t base = ((size_t)hk * a.L_max + (size_t)ct * BKEY) * D;
-                load_tile(smem + i * STAGE_BYTES, a.k_cache + base, a.v_cache + base, D, min(BKEY, rg.L - ct * BKEY));
-            }
-            cp_async_commit();
-        }
-    };
-    prefetch_cache_tiles();
-    prefetch_weights(a.pf, (((long long)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * THREADS + threadIdx.x,
-                     (long long)gridDim.x * gridDim.y * gridDim.z * THREADS);
-    pdl_wait();
-    {
-        const int L_now = min(max(*a.cache_len, 0), a.L_max);
-        if (L_now != rg.L) {
-            cp_async_wait<0>();
-            __syncthreads();
-            rg = plan_ranges(a, L_now, sp);
-            prefetch_cache_tiles();
-        }
-    }
-    const int L = rg.L, nt = rg.nt;
-    if (rg.rows_mode) {
-        if (sp < 2)
-            attention_rows_mode(a, smem_all, h, sp, L, nt);
-        return;
-    }
-    if (rg.idle)
-        return;
-    const int n_active = rg.n_active, tile0 = rg.tile0, tile1 = rg.tile1, n_tiles = rg.n_tiles;
 
     auto issue = [&](int i) {
-        // tile i of this CTA: a cache tile, or (last, if this is the last range) the tree's own keys
+        // tile i of this CTA: a cache tile, or (last, if has_tree) the tree's own keys
         uint8_t *stage = smem + (i % STAGES) * STAGE_BYTES;
         const int ct = tile0 + i;
         if (ct < tile1) {
             const size_t base = ((size_t)hk * a.L_max + (size_t)ct * BKEY) * D;
             load_tile(stage, a.k_cache + base, a.v_cache + base, D, min(BKEY, L - ct * BKEY));
         } else {
-            const int w = ct - tile1;  // key tile of the tree
-            const size_t base = ((size_t)w * BKEY * a.Hkv + hk) * D;
-            load_tile(stage, a.k_new + base, a.v_new + base, HkvD, min(BKEY, a.T - w * BKEY));
+            const int w = LARGE ? ct - tile1 : 0;  // key tile of the tree
+            const size_t tb = ((size_t)w * BKEY * a.Hkv + hk) * D;
+            load_tile(stage, a.k_new + tb, a.v_new + tb, HkvD, min(BKEY, a.T - w * BKEY));
         }
     };
-    // ---- after the wait: Q, and the tree's own tiles that are among the first STAGES-1 tiles, as one more copy group
+    // ---- Q and the first K/V tiles are requested together; Q is copy group 0
     {
         const uint32_t qb = smem_u32(smem_all);
 #pragma unroll
@@ -445,19 +403,21 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             int r = idx >> 4, c = idx & 15;
             bool ok = r < Tq;
             cp_async16(qb + tile_off(r, c), a.q + (size_t)(ok ? q0 + r : 0) * HD + (size_t)h * D + c * 8, ok);
-            if (has_qlo)
+            if (QLO)
                 cp_async16(qb + TILE_BYTES + tile_off(r, c), a.q_lo + (size_t)(ok ? q0 + r : 0) * HD + (size_t)h * D + c * 8, ok);
         }
-        for (int i = 0; i < STAGES - 1; ++i)
-            if (i < n_tiles && tile0 + i >= tile1)
-                issue(i);
         cp_async_commit();
     }
-    cp_async_wait<0>();  // Q and the first STAGES-1 tiles have landed
+    for (int i = 0; i < STAGES - 1; ++i) {
+        if (i < n_tiles)
+            issue(i);
+        cp_async_commit();
+    }
+    cp_async_wait<STAGES - 1>();  // everything but the K/V groups just issued: Q has landed
     __syncthreads();
     uint32_t qf[8][4];
     const int q_row = wq * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
-    const uint32_t q_lo_addr = smem_u32(smem_all) + TILE_BYTES;
+    const uint32_t q_lo_addr = smem_u32(smem_all) + TILE_BYTES;  // second plane's tile (QLO): fragments are re-read per tile
     {
         const uint32_t qb = smem_u32(smem_all);
 #pragma unroll
@@ -466,6 +426,11 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     }
 
     const int row0 = wq * 16 + g, row1 = row0 + 8;  // rows inside the query tile
+    // mask words of this thread's two rows for the tree's first key tile; with LARGE the words of the following key tiles
+    // are fetched one tile ahead inside the loop
+    uint64_t mask0 = row0 < Tq ? a.mask[(size_t)(q0 + row0) * (LARGE ? a.mask_words : 1)] : 0ull;
+    uint64_t mask1 = row1 < Tq ? a.mask[(size_t)(q0 + row1) * (LARGE ? a.mask_words : 1)] : 0ull;
+    uint64_t next_mask0 = 0ull, next_mask1 = 0ull;
     const float sc = rsqrtf((float)D) * LOG2E;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     float o[16][4];
@@ -491,7 +456,7 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t ql[4];
-            if (has_qlo)  // the second plane's fragments come from shared memory: no registers to hold them
+            if (QLO)  // the second plane's fragments come from shared memory: there are no registers to hold them
                 ldsm_x4(q_lo_addr + tile_off(q_row, 2 * ks + (lane >> 4)), ql[0], ql[1], ql[2], ql[3]);
 #pragma unroll
             for (int np = 0; np < 2; ++np) {
@@ -500,7 +465,7 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
                 ldsm_x4(kb + tile_off(kr, 2 * ks + ((lane >> 3) & 1)), b0, b1, b2, b3);
                 mma_bf16(s[2 * np], qf[ks], b0, b1);
                 mma_bf16(s[2 * np + 1], qf[ks], b2, b3);
-                if (has_qlo) {
+                if (QLO) {
                     mma_bf16(s[2 * np], ql, b0, b1);
                     mma_bf16(s[2 * np + 1], ql, b2, b3);
                 }
@@ -509,12 +474,14 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
         // ---- mask + online softmax (log2 domain)
         float mx0 = -INFINITY, mx1 = -INFINITY;
         const int key_base = ct * BKEY;
-        // a tree tile: this thread's two query rows' mask words for that key tile (ancestors inside keys 64 w .. 64 w + 63)
-        uint64_t mask0 = 0ull, mask1 = 0ull;
-        if (tree_tile) {
+        if (LARGE && tree_tile) {
+            // this key tile's words were fetched a tile ago (the first one before the loop); ask for the next tile's now
             const int w = ct - tile1;
-            if (row0 < Tq) mask0 = a.mask[(size_t)(q0 + row0) * a.mask_words + w];
-            if (row1 < Tq) mask1 = a.mask[(size_t)(q0 + row1) * a.mask_words + w];
+            if (w > 0) { mask0 = next_mask0; mask1 = next_mask1; }
+            if (w + 1 < tree_tiles) {
+                if (row0 < Tq) next_mask0 = a.mask[(size_t)(q0 + row0) * a.mask_words + w + 1];
+                if (row1 < Tq) next_mask1 = a.mask[(size_t)(q0 + row1) * a.mask_words + w + 1];
+            }
         }
 #pragma unroll
         for (int n = 0; n < 4; ++n) {
@@ -653,7 +620,6 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
         return;
     }
     // ---- partial result of this key range
-    const size_t slot = (size_t)blockIdx.z * a.H + h;  // (query tile, head)
     float *wo = a.ws_o + (slot * a.max_splits + sp) * BQ * D;
     float *wml = a.ws_ml + (slot * a.max_splits + sp) * 2 * BQ;
     if (owner) {
@@ -676,72 +642,78 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     __syncthreads();
     if (s_ticket != n_active - 1)
         return;
-    // ---- last CTA of this head: combine the key ranges in range order.  Thread -> 4 adjacent columns of 8 rows.  Every
-    // thread reads its rows' (max, sum) records itself (the lanes of a warp read the same 64 bytes: one broadcast
-    // transaction) together with the partial outputs, two ranges per round, all loads of a round in flight at once, and
-    // folds them in with a running maximum: one trip to the L2 instead of a staged max / weight / output sequence.
+    // ---- last CTA of this head: combine the key ranges in split order
     __threadfence();
+    float (*s_w)[BQ] = reinterpret_cast<float (*)[BQ]>(smem);  // [max_splits + 1][64] weights; the ring is idle now
+    float *s_ml = reinterpret_cast<float *>(smem) + (FLASH_MAX_SPLITS + 1) * BQ;  // staged (max, sum) pairs [split][2][64]
     const float *__restrict__ mlh = a.ws_ml + slot * a.max_splits * 2 * BQ;
+    {
+        // one batch of independent loads: thread t fetches element t of every key range's 128-float record
+        float t[FLASH_MAX_SPLITS];
+        const bool mine = threadIdx.x < 2 * BQ;
+#pragma unroll
+        for (int s2 = 0; s2 < FLASH_MAX_SPLITS; ++s2)
+            if (mine && s2 < n_active) t[s2] = mlh[(size_t)s2 * 2 * BQ + threadIdx.x];
+#pragma unroll
+        for (int s2 = 0; s2 < FLASH_MAX_SPLITS; ++s2)
+            if (mine && s2 < n_active) s_ml[s2 * 2 * BQ + threadIdx.x] = t[s2];
+    }
+    __syncthreads();
+    if (threadIdx.x < BQ) {
+        const int r = threadIdx.x;
+        float mstar = -INFINITY;
+        for (int s2 = 0; s2 < n_active; ++s2)
+            mstar = fmaxf(mstar, s_ml[s2 * 2 * BQ + r]);
+        const float msafe = mstar == -INFINITY ? 0.f : mstar;
+        float lstar = 0.f;
+        for (int s2 = 0; s2 < n_active; ++s2) {
+            const float w = exp2f(s_ml[s2 * 2 * BQ + r] - msafe);
+            s_w[s2][r] = w;
+            lstar += w * s_ml[s2 * 2 * BQ + BQ + r];
+        }
+        s_w[FLASH_MAX_SPLITS][r] = lstar > 0.f ? 1.0f / lstar : 0.f;
+        if (a.lse && r < Tq)
+            a.lse[(size_t)(q0 + r) * a.H + h] = mstar / LOG2E + logf(lstar);
+    }
+    __syncthreads();
+    // thread -> 4 adjacent columns of 8 rows; per key range the 8 row loads are in flight together
     const float *__restrict__ oh = a.ws_o + slot * a.max_splits * BQ * D;
-    const int c4 = (threadIdx.x & 31) * 4, r8 = (threadIdx.x >> 5) * 8;
-    float mrun[8], lrun[8];
+    const int c4 = (threadIdx.x & 31) * 4, rg = (threadIdx.x >> 5) * 8;
     float4 acc[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        mrun[u] = -INFINITY;
-        lrun[u] = 0.f;
+    for (int u = 0; u < 8; ++u)
         acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     for (int s2 = 0; s2 < n_active; s2 += 2) {
+        // two key ranges (16 independent 16-byte loads per thread) in flight per round; always added in range order
+        float4 v[8], v2[8];
         const bool two = s2 + 1 < n_active;
-        float4 v[8], v2[8], pm[2], pl[2], qm[2], ql[2];
-        const float *rec = mlh + (size_t)s2 * 2 * BQ;
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            pm[u] = *reinterpret_cast<const float4 *>(rec + r8 + 4 * u);
-            pl[u] = *reinterpret_cast<const float4 *>(rec + BQ + r8 + 4 * u);
-        }
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            v[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)s2 * BQ + r8 + u) * D + c4);
+            v[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)s2 * BQ + rg + u) * D + c4);
         if (two) {
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                qm[u] = *reinterpret_cast<const float4 *>(rec + 2 * BQ + r8 + 4 * u);
-                ql[u] = *reinterpret_cast<const float4 *>(rec + 3 * BQ + r8 + 4 * u);
-            }
-#pragma unroll
             for (int u = 0; u < 8; ++u)
-                v2[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)(s2 + 1) * BQ + r8 + u) * D + c4);
+                v2[u] = *reinterpret_cast<const float4 *>(oh + ((size_t)(s2 + 1) * BQ + rg + u) * D + c4);
         }
-        const float *pmf = reinterpret_cast<const float *>(pm), *plf = reinterpret_cast<const float *>(pl);
-        const float *qmf = reinterpret_cast<const float *>(qm), *qlf = reinterpret_cast<const float *>(ql);
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const float ma = pmf[u], mb = two ? qmf[u] : -INFINITY;
-            const float mn = fmaxf(mrun[u], fmaxf(ma, mb));
-            const float ms = mn == -INFINITY ? 0.f : mn;
-            const float c = exp2f(mrun[u] - ms), wa = exp2f(ma - ms), wb = exp2f(mb - ms);  // exp2f(-inf) = 0
-            mrun[u] = mn;
-            lrun[u] = lrun[u] * c + wa * plf[u] + (two ? wb * qlf[u] : 0.f);
-            acc[u].x = acc[u].x * c + wa * v[u].x;
-            acc[u].y = acc[u].y * c + wa * v[u].y;
-            acc[u].z = acc[u].z * c + wa * v[u].z;
-            acc[u].w = acc[u].w * c + wa * v[u].w;
-            if (two) {
-                acc[u].x += wb * v2[u].x;
-                acc[u].y += wb * v2[u].y;
-                acc[u].z += wb * v2[u].z;
-                acc[u].w += wb * v2[u].w;
+            const float w = s_w[s2][rg + u];
+            acc[u].x += w * v[u].x; acc[u].y += w * v[u].y; acc[u].z += w * v[u].z; acc[u].w += w * v[u].w;
+        }
+        if (two) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float w = s_w[s2 + 1][rg + u];
+                acc[u].x += w * v2[u].x; acc[u].y += w * v2[u].y; acc[u].z += w * v2[u].z; acc[u].w += w * v2[u].w;
             }
         }
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-        const int r = r8 + u;
+        const int r = rg + u;
         if (r >= Tq)
             continue;
-        const float inv = lrun[u] > 0.f ? 1.0f / lrun[u] : 0.f;
+        const float inv = s_w[FLASH_MAX_SPLITS][r];
         const float y[4] = {acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv};
         const size_t idx = (size_t)(q0 + r) * HD + (size_t)h * D + c4;
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]), h1 = __floats2bfloat162_rn(y[2], y[3]);
@@ -756,8 +728,6 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             pk.y = *reinterpret_cast<const uint32_t *>(&q1);
             *reinterpret_cast<uint2 *>(a.out_lo + idx) = pk;
         }
-        if (a.lse && c4 == 0)
-            a.lse[(size_t)(q0 + r) * a.H + h] = mrun[u] / LOG2E + logf(lrun[u]);
     }
     if (threadIdx.x == 0)
         a.counters[slot] = 0;  // ready for the next launch
@@ -772,21 +742,40 @@ static int rows_mode_max_tiles()
     return v;
 }
 
-static bool g_flash_attr_set[64] = {};  // devices on which the kernel's shared-memory limit has been raised
-
 size_t tree_attention_flash_workspace_bytes(int H, int q_tiles)
 {
     const size_t slots = (size_t)H * (q_tiles > 0 ? q_tiles : 1);
     return slots * FLASH_MAX_SPLITS * (BQ * D + 2 * BQ) * sizeof(float) + slots * sizeof(int);
 }
 
+// The kernel's instantiations and their dynamic shared memory; the limit is raised once per device.
+typedef void (*FlashKernel)(Args);
+static FlashKernel flash_kernel(bool qlo, bool large)
+{
+    return qlo ? (large ? tree_attention_flash_kernel<true, true> : tree_attention_flash_kernel<true, false>)
+               : (large ? tree_attention_flash_kernel<false, true> : tree_attention_flash_kernel<false, false>);
+}
+static cudaError_t flash_set_limits()
+{
+    static bool done[64] = {};
+    if (!first_use_on_current_device(done))
+        return cudaSuccess;
+    for (int q = 0; q < 2; ++q)
+        for (int l = 0; l < 2; ++l) {
+            cudaError_t e = cudaFuncSetAttribute(flash_kernel(q, l), cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(q));
+            if (e != cudaSuccess)
+                return e;
+        }
+    return cudaSuccess;
+}
+
 cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                        int L_hint, cudaStream_t s, const void *q_lo, const WeightPrefetch *prefetch, int mask_words)
+                                        int L_hint, cudaStream_t s, const void *q_lo, int mask_words)
 {
-    if (first_use_on_current_device(g_flash_attr_set)) {
-        cudaError_t e = cudaFuncSetAttribute(tree_attention_flash_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    {
+        cudaError_t e = flash_set_limits();
         if (e != cudaSuccess)
             return e;
     }
@@ -805,22 +794,21 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
         }
     }
     Args a;
+    const int q_tiles = (T + BQ - 1) / BQ;
+    const bool large = q_tiles > 1, qlo = q_lo != nullptr;
+    const size_t slots = (size_t)H * q_tiles;
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
     a.q_lo = (const bf16 *)q_lo;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
-    a.cache_len = cache_len; a.mask = mask; a.out = (bf16 *)out; a.out_lo = (bf16 *)out_lo; a.lse = lse;
-    const int q_tiles = (T + BQ - 1) / BQ;
-    const size_t slots = (size_t)H * q_tiles;
+    a.cache_len = cache_len; a.mask = mask; a.mask_words = mask_words > 0 ? mask_words : 1;
+    a.out = (bf16 *)out; a.out_lo = (bf16 *)out_lo; a.lse = lse;
     a.ws_o = (float *)workspace;
     a.ws_ml = a.ws_o + slots * FLASH_MAX_SPLITS * BQ * D;
     a.counters = (int *)(a.ws_ml + slots * FLASH_MAX_SPLITS * 2 * BQ);
-    a.mask_words = mask_words > 0 ? mask_words : 1;
-    a.q_tiles = q_tiles;
     a.T = T; a.H = H; a.Hkv = Hkv; a.L_max = L_max; a.tiles_per_split = tps; a.max_splits = FLASH_MAX_SPLITS;
     a.rows_max_tiles = rows_mode_max_tiles();
-    a.pf = prefetch ? *prefetch : WeightPrefetch{};
     dim3 grid(H, splits, q_tiles);
-    launch_pdl(tree_attention_flash_kernel, dim3(grid), dim3(THREADS), SMEM_BYTES, s, a);
+    launch_pdl(flash_kernel(qlo, large), dim3(grid), dim3(THREADS), (size_t)smem_bytes(qlo), s, a);
     return cudaGetLastError();
 }
 
@@ -884,7 +872,7 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
             fprintf(stderr, "medusa_tree_attention_static: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
             return MEDUSA_ERR_CUDA;
         }
-        e = cudaFuncSetAttribute(tree_attention_flash_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        e = flash_set_limits();
         if (e != cudaSuccess) {
             fprintf(stderr, "medusa_tree_attention_static: cudaFuncSetAttribute failed: %s\n", cudaGetErrorString(e));
             return MEDUSA_ERR_CUDA;
@@ -897,7 +885,7 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
     a.q_lo = nullptr;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
-    a.cache_len = cache_len; a.mask = mask; a.out = (bf16 *)out; a.out_lo = nullptr; a.lse = lse;
+    a.cache_len = cache_len; a.mask = mask; a.mask_words = 1; a.out = (bf16 *)out; a.out_lo = nullptr; a.lse = lse;
     a.ws_o = base;
     a.ws_ml = base + STATIC_O_FLOATS;
     a.counters = (int *)(base + STATIC_O_FLOATS + STATIC_ML_FLOATS);
@@ -913,11 +901,8 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
         tps = (nt + STATIC_MAX_SPLITS - 1) / STATIC_MAX_SPLITS;
         splits = (nt + tps - 1) / tps;
     }
-    a.mask_words = 1;
-    a.q_tiles = 1;
     a.T = T; a.H = H; a.Hkv = H; a.L_max = L_max; a.tiles_per_split = tps; a.max_splits = STATIC_MAX_SPLITS;
     a.rows_max_tiles = rows_mode_max_tiles();
-    a.pf = WeightPrefetch{};
-    cudaError_t e = launch_pdl(tree_attention_flash_kernel, dim3(H, splits), dim3(THREADS), (size_t)SMEM_BYTES, s, a);
+    cudaError_t e = launch_pdl(flash_kernel(false, false), dim3(H, splits), dim3(THREADS), (size_t)smem_bytes(false), s, a);
     return e == cudaSuccess ? MEDUSA_OK : MEDUSA_ERR_CUDA;
 }

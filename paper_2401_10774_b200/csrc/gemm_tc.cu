@@ -40,8 +40,9 @@ constexpr int UMMA_K = 16;
 constexpr int MAX_STAGES = 8;         // ring depth is a launch parameter (a.stages)
 constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;    // 8 KiB per plane
-constexpr int STAGE_BYTES = A_BYTES + 2 * B_BYTES;
-constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */; }
+// a stage: one weight tile and, for each of the launch's RT token tiles, the two activation planes
+constexpr int stage_bytes(int rt) { return A_BYTES + rt * 2 * B_BYTES; }
+constexpr int smem_bytes(int stages, int rt) { return stages * stage_bytes(rt) + 1024 /* alignment slack */ + 256 /* barriers */; }
 constexpr int THREADS = 192;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -192,10 +193,18 @@ struct SegmentIter {
     }
 };
 
-__global__ void __launch_bounds__(THREADS, 2)
+// RT = token tiles (64 rows each) per launch.  RT = 1: two CTAs per SM, two 128-column accumulators each.  RT = 2 (trees
+// of more than 64 nodes): the weight tile of a stage feeds two MMAs, one per token tile, into two accumulators; a CTA then
+// holds all 512 tensor-memory columns (2 buffers x 2 tiles x 128), so one CTA per SM with a deeper ring.
+template <int RT>
+__global__ void __launch_bounds__(THREADS, RT == 1 ? 2 : 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW0,
                const __grid_constant__ CUtensorMap mapW1, const __grid_constant__ CUtensorMap mapW2, GemmTcArgs a)
 {
+    constexpr int STAGE_BYTES = stage_bytes(RT);
+    constexpr uint32_t ACC_COLS = RT * UMMA_N;   // columns of one accumulator set (all token tiles of a segment)
+    const int rt_n = min(RT, (a.T + BN - 1) / BN);  // token tiles that hold rows in this launch
+    const uint32_t stage_tx = (uint32_t)(A_BYTES + rt_n * 2 * B_BYTES);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the next kernel may start its prologue
     extern __shared__ uint8_t smem_raw[];
     // tiles must sit on 1024-byte boundaries for the 128-byte swizzle pattern
@@ -223,7 +232,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
     uint32_t tmem_base = 0;
     if (warp != 0) {
         if (warp == 1) {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(2 * UMMA_N));
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(2 * ACC_COLS));
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -238,6 +247,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             uint64_t pol_stream, pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            // the activation planes of k block `k` for every token tile of the launch: hi rows, then lo rows
+            auto load_x = [&](uint8_t *st, int k, uint64_t *bar) {
+                for (int rt = 0; rt < rt_n; ++rt) {
+                    tma_load_2d(st + A_BYTES + rt * 2 * B_BYTES, &mapX, k, a.x_row_hi + rt * BN, bar, pol_keep);
+                    tma_load_2d(st + A_BYTES + rt * 2 * B_BYTES + B_BYTES, &mapX, k, a.x_row_lo + rt * BN, bar, pol_keep);
+                }
+            };
             SegmentIter it(a, blockIdx.x);
             Segment sg;
             int n = 0;          // k blocks issued so far by this CTA
@@ -259,11 +275,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                             // the ring is full of weight tiles: now wait for the producer of X, then add the X tiles
                             asm volatile("griddepcontrol.wait;" ::: "memory");
                             waited = true;
-                            for (int p = 0; p < pend_n; ++p) {
-                                uint8_t *st = tiles + p * STAGE_BYTES;
-                                tma_load_2d(st + A_BYTES, &mapX, pend_k[p], a.x_row_hi, &sm->full[p], pol_keep);
-                                tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], a.x_row_lo, &sm->full[p], pol_keep);
-                            }
+                            for (int p = 0; p < pend_n; ++p)
+                                load_x(tiles + p * STAGE_BYTES, pend_k[p], &sm->full[p]);
                         }
                         if (sm->failed || !mbar_wait(&sm->empty[s], ph, a.spin_limit)) {
                             sm->failed = 1;
@@ -273,11 +286,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     }
                     uint8_t *st = tiles + s * STAGE_BYTES;
                     const int k = (sg.kb0 + i) * BK;
-                    mbar_expect_tx(&sm->full[s], STAGE_BYTES);
+                    mbar_expect_tx(&sm->full[s], stage_tx);
                     tma_load_2d(st, mapW, k, trow, &sm->full[s], pol_stream);
                     if (waited) {
-                        tma_load_2d(st + A_BYTES, &mapX, k, a.x_row_hi, &sm->full[s], pol_keep);
-                        tma_load_2d(st + A_BYTES + B_BYTES, &mapX, k, a.x_row_lo, &sm->full[s], pol_keep);
+                        load_x(st, k, &sm->full[s]);
                     } else {
                         pend_k[pend_n++] = k;  // n < STAGES here, so stage index == pend index
                     }
@@ -289,11 +301,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             }
             if (!waited && ok) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
-                for (int p = 0; p < pend_n; ++p) {
-                    uint8_t *st = tiles + p * STAGE_BYTES;
-                    tma_load_2d(st + A_BYTES, &mapX, pend_k[p], a.x_row_hi, &sm->full[p], pol_keep);
-                    tma_load_2d(st + A_BYTES + B_BYTES, &mapX, pend_k[p], a.x_row_lo, &sm->full[p], pol_keep);
-                }
+                for (int p = 0; p < pend_n; ++p)
+                    load_x(tiles + p * STAGE_BYTES, pend_k[p], &sm->full[p]);
             }
         }
     } else if (warp == 1) {
@@ -312,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     break;
                 }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");  // the epilogue has drained this accumulator
-                const uint32_t tmem_d = tmem_base + (uint32_t)(b * UMMA_N);
+                const uint32_t tmem_d = tmem_base + (uint32_t)b * ACC_COLS;
                 for (int i = 0; i < sg.nkb; ++i) {
                     if (sm->failed || !mbar_wait(&sm->full[st], ph, a.spin_limit)) {
                         sm->failed = 1;
@@ -320,12 +329,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                         break;
                     }
                     const uint32_t sa = smem_u32(tiles + st * STAGE_BYTES);
-                    // the two activation planes sit back to back in the stage: one 128-row K-major operand
-                    const uint64_t da = umma_desc(sa), db = umma_desc(sa + A_BYTES);
+                    // the two activation planes of a token tile sit back to back in the stage: one 128-row K-major operand
+                    const uint64_t da = umma_desc(sa);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t adv = (uint64_t)((k * UMMA_K * 2) >> 4);  // 32 bytes per step inside the swizzled row
-                        umma(tmem_d, da + adv, db + adv, (i | k) ? 1u : 0u, leader);
+                    for (int rt = 0; rt < RT; ++rt) {
+                        if (rt < rt_n) {
+                            const uint64_t db = umma_desc(sa + A_BYTES + rt * 2 * B_BYTES);
+#pragma unroll
+                            for (int k = 0; k < BK / UMMA_K; ++k) {
+                                const uint64_t adv = (uint64_t)((k * UMMA_K * 2) >> 4);  // 32 bytes per step inside the swizzled row
+                                umma(tmem_d + (uint32_t)(rt * UMMA_N), da + adv, db + adv, (i | k) ? 1u : 0u, leader);
+                            }
+                        }
                     }
                     umma_commit(&sm->empty[st], leader);  // frees the stage once these MMAs have read it
                     if (++st == STAGES) {
@@ -359,26 +374,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             const bool n_ok = n < (seg == 0 ? a.seg0_cols : a.seg_cols);
             // columns t (W * X_hi) and 64 + t (W * X_lo) of the same lane add up to the result for token t; both
             // loads of a half are in flight together, and a full 64-row store runs without per-row tests
-            const bool all_rows = a.row0 == 0 && a.T == BN;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t v[32], w[32];
-                const uint32_t col = (uint32_t)(b * UMMA_N + half * 32);
-                tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col, v);
-                tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col + BN, w);
-                tmem_ld_wait();
-                if (n_ok) {
-                    float *o = out + (size_t)(half * 32) * a.ldy;  // a warp writes 32 consecutive floats per token row
-                    if (all_rows) {
+            for (int rt = 0; rt < RT; ++rt) {
+                if (rt >= rt_n)
+                    break;
+                const int tb = rt * BN;  // first token row of this tile inside the launch
+                const bool all_rows = a.row0 <= tb && a.T >= tb + BN;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i, o += a.ldy)
-                            *o = __uint_as_float(v[i]) + __uint_as_float(w[i]);
-                    } else {
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t v[32], w[32];
+                    const uint32_t col = (uint32_t)b * ACC_COLS + (uint32_t)(rt * UMMA_N + half * 32);
+                    tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col, v);
+                    tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col + BN, w);
+                    tmem_ld_wait();
+                    if (n_ok) {
+                        float *o = out + (size_t)(tb + half * 32) * a.ldy;  // a warp writes 32 consecutive floats per token row
+                        if (all_rows) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i, o += a.ldy) {
-                            const int t = half * 32 + i;
-                            if (t >= a.row0 && t < a.T)
+                            for (int i = 0; i < 32; ++i, o += a.ldy)
                                 *o = __uint_as_float(v[i]) + __uint_as_float(w[i]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i, o += a.ldy) {
+                                const int t = tb + half * 32 + i;
+                                if (t >= a.row0 && t < a.T)
+                                    *o = __uint_as_float(v[i]) + __uint_as_float(w[i]);
+                            }
                         }
                     }
                 }
@@ -405,7 +426,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         __syncthreads();
     }
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * UMMA_N));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * ACC_COLS));
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -463,7 +484,12 @@ int gemm_tc_stages()
     return v;
 }
 
-int gemm_tc_num_ctas()
+// Token tiles per launch: one for up to 64 rows, two for more (the weight stream then serves both tiles).
+int gemm_tc_row_tiles(int T) { return T > BN ? 2 : 1; }
+// ring depth of the two-tile form (one CTA per SM, 48 KiB per stage)
+static int gemm_tc_stages_rt2() { return 4; }
+
+int gemm_tc_num_ctas(int row_tiles)
 {
     static int sms = 0;
     if (!sms) {
@@ -472,17 +498,17 @@ int gemm_tc_num_ctas()
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             sms = 148;
     }
-    return sms * gemm_tc_ctas_per_sm();
+    return sms * (row_tiles > 1 ? 1 : gemm_tc_ctas_per_sm());
 }
 
-PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols)
+PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols, int row_tiles)
 {
     PlaneDesc pd{};
     if (seg0_cols <= 0) seg0_cols = seg_cols;
     const int tiles = (seg0_cols + BM - 1) / BM + (n_seg - 1) * ((seg_cols + BM - 1) / BM);
     const int KB = (K + BK - 1) / BK;
     const long long total = (long long)tiles * KB;
-    int G = gemm_tc_num_ctas();
+    int G = gemm_tc_num_ctas(row_tiles);
     if (whole_tiles) {
         if (G > tiles) G = tiles;
         pd.n_max = 1; pd.KB = KB; pd.G = 0; pd.total = total; pd.stride = plane_stride; pd.ctas = G;
@@ -498,39 +524,17 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
     return pd;
 }
 
-WeightPrefetch gemm_tc_prefetch_plan(const void *const *W, int n_seg, int seg_cols, int K, bool whole_tiles, int seg0_cols,
-                                     int units)
-{
-    WeightPrefetch p{};
-    if (seg0_cols <= 0) seg0_cols = seg_cols;
-    if (K % BK != 0 || units <= 0 || !W)
-        return p;  // units = 0
-    const PlaneDesc pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, 0, seg0_cols);
-    for (int i = 0; i < 3; ++i) p.W[i] = W[i < n_seg ? i : 0];
-    p.n_seg = n_seg;
-    p.seg0_tiles = (seg0_cols + BM - 1) / BM;
-    p.seg_tiles = (seg_cols + BM - 1) / BM;
-    p.seg0_rows = seg0_cols;
-    p.seg_rows = seg_cols;
-    p.K = K;
-    p.KB = pd.KB;
-    p.G = pd.ctas;
-    p.whole_tiles = whole_tiles ? 1 : 0;
-    p.total = pd.total;
-    // never more than a CTA's whole range (the prefetching threads walk G * units * 128 rows)
-    const long long per_cta = p.whole_tiles ? p.KB : (pd.total + p.G - 1) / p.G;
-    p.units = (long long)units < per_cta ? units : (int)per_cta;
-    return p;
-}
-
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo)
+                           int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo, int row_tiles)
 {
     if (seg0_cols <= 0) seg0_cols = seg_cols;
+    const int stages = row_tiles > 1 ? gemm_tc_stages_rt2() : gemm_tc_stages();
     static bool attr_set[64] = {};
     if (first_use_on_current_device(attr_set)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(gemm_tc_stages()));
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(gemm_tc_stages(), 1));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(gemm_tc_stages_rt2(), 2));
         if (e != cudaSuccess)
             return e;
     }
@@ -549,7 +553,7 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     a.T = T;
     a.row0 = row0;
     a.status = status;
-    a.stages = gemm_tc_stages();
+    a.stages = stages;
     a.spin_limit = spin_limit ? spin_limit : DEFAULT_SPIN_LIMIT;
     a.withhold = withhold;
     a.x_row_hi = x_row_hi;
@@ -560,14 +564,16 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(pd.ctas);
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = smem_bytes(a.stages);
+    cfg.dynamicSmemBytes = smem_bytes(a.stages, row_tiles > 1 ? 2 : 1);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = tuning_env("MEDUSA_NO_PDL") ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
+    if (row_tiles > 1)
+        return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1>, *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
 }
 
 }  // namespace medusa

@@ -56,34 +56,26 @@ struct GemmTcArgs {
     int x_row_hi, x_row_lo;  // rows of the activation tensor where this launch's 64 token rows start in the hi / lo plane
 };
 
-// What a kernel that runs before a projection launch needs to know to pull that launch's first weight tiles into the
-// L2 (prefetch.cuh).  units == 0: nothing to prefetch.
-struct WeightPrefetch {
-    const void *W[3];        // weight matrices of the launch ([rows][K] bf16)
-    int n_seg, seg0_tiles, seg_tiles, seg0_rows, seg_rows;
-    int K, KB, G, whole_tiles;
-    long long total;         // tiles * KB
-    int units;               // (tile, k block) pairs per CTA to prefetch
-};
-// plan of the prefetch for a launch described like gemm_tc_plan's; K must be a multiple of 64 (else units = 0)
-WeightPrefetch gemm_tc_prefetch_plan(const void *const *W, int n_seg, int seg_cols, int K, bool whole_tiles, int seg0_cols,
-                                     int units);
-
 // W: [N][K] bf16 row-major
 bool make_weight_map(TensorMap *out, const void *W, int N, int K);
 // X_planes: split activation, [2][rows][K] bf16 (hi plane, then lo plane; rows a multiple of 64)
 bool make_act_map(TensorMap *out, const void *X_planes, int K, int rows = 64);
-int gemm_tc_num_ctas();
+int gemm_tc_num_ctas(int row_tiles = 1);
+// token tiles (64 rows each) one launch covers for a pass over T rows: 1 up to 64 rows, 2 beyond
+int gemm_tc_row_tiles(int T);
 int gemm_tc_stages();
 int gemm_tc_ctas_per_sm();
 // plan of a launch over n_seg weight matrices of seg_cols rows (seg_cols % 128 == 0 unless n_seg == 1); the first
 // matrix has seg0_cols rows if that is given (> 0, a multiple of 128)
-PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols = 0);
+PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols = 0,
+                       int row_tiles = 1);
 // P[piece][t][first column of segment seg + n] = partial sums over k of (X_hi + X_lo)[t][k] * W_seg[n][k], t in [row0, T);
-// the launch's token rows t = 0..63 are rows x_row_hi + t and x_row_lo + t of the activation tensor (a tree of more
-// than 64 tokens is projected in tiles of 64 rows, one launch each, with P advanced by 64 rows)
+// the launch's token rows t = 0.. are rows x_row_hi + t and x_row_lo + t of the activation tensor: 64 rows per launch
+// with row_tiles = 1, 128 with row_tiles = 2 (pd must come from gemm_tc_plan with the same row_tiles); a tree of more
+// rows than one launch covers is projected launch by launch with P advanced accordingly
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0, int x_row_hi = 0, int x_row_lo = 64);
+                           int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0, int x_row_hi = 0, int x_row_lo = 64,
+                           int row_tiles = 1);
 
 }  // namespace medusa

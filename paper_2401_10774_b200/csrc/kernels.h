@@ -16,14 +16,11 @@ void launch_embed(int dtype, const int32_t *tok, const void *embed, float *x, in
 // hi = bf16(y) and lo = bf16(y - hi); a product with bf16 weights is then W*hi + W*lo, accurate to ~2^-17.
 // In the f32 model there is one float plane and lo is null.
 // out/out_lo: [T][d] planes (out_lo nullable); out_f32 (nullable): the unrounded values
-// `prefetch` (nullable) on a launcher: the weight tiles of the projection that follows, which the kernel's threads ask
-// the L2 for before they wait for their own input (prefetch.cuh).
 // Projections write partial results as float planes (PlaneDesc, gemm_tc.h); the kernels below that consume
 // them add a column's planes in order before anything else.
 // x (+= sum of planes, written back if pd.n_max > 0), then RMSNorm(x) -> out planes
 void launch_add_rmsnorm(int dtype, float *x, const float *planes, const PlaneDesc &pd, const void *gain,
-                        float eps, void *out, void *out_lo, float *out_f32, int T, int d, cudaStream_t s,
-                        const WeightPrefetch *prefetch = nullptr);
+                        float eps, void *out, void *out_lo, float *out_f32, int T, int d, cudaStream_t s);
 // Y[t][col0 + n] (float, row stride ldy) (+)= sum_k (X[t][k] + Xlo[t][k]) * W[n][k];  X planes [T][K], row stride ldx
 void launch_gemm_simt(int dtype, const void *X, const void *Xlo, int ldx, const void *W, void *Y, int ldy, int col0,
                       int T, int N, int K, GemmOut mode, cudaStream_t s);
@@ -39,7 +36,7 @@ void launch_rope_split(int dtype, const float *qkv, const PlaneDesc &pd_q, const
 void launch_rope_apply(int dtype, const void *in, const float2 *cs, void *out, int T, int H, int D, cudaStream_t s);
 // gate_up float [T][2F] -> act[t][i] = SiLU(gate) * up, rounded once to the activation dtype
 void launch_silu_mul(int dtype, const float *gate_up, const PlaneDesc &pd, void *act, void *act_lo, int T,
-                     int F, cudaStream_t s, const WeightPrefetch *prefetch = nullptr);
+                     int F, cudaStream_t s);
 
 // sums `bytes` bytes with 16-byte streaming loads (a pure DRAM read stream); sink: >= blocks floats
 void launch_stream_read(const void *buf, long long bytes, float *sink, int blocks, cudaStream_t s);
@@ -64,8 +61,7 @@ size_t tree_attention_flash_workspace_bytes(int H, int q_tiles = 1);  // q_tiles
 cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                        int L_hint, cudaStream_t s, const void *q_lo = nullptr,
-                                        const WeightPrefetch *prefetch = nullptr, int mask_words = 1);
+                                        int L_hint, cudaStream_t s, const void *q_lo = nullptr, int mask_words = 1);
 // The same operation and workspace on the tcgen05 tensor cores (attention_tc.cu): scores and P V accumulate in
 // TMEM, softmax threads own one query row each.  status: device status word (MEDUSA_ERR_TIMEOUT on an expired wait).
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,

@@ -5,7 +5,6 @@
 #include "common.cuh"
 #include "pdl.cuh"
 #include "kernels.h"
-#include "prefetch.cuh"
 
 namespace medusa {
 
@@ -125,11 +124,9 @@ template <typename WT, int GROUPS, int MAXT>
 __global__ void __launch_bounds__(MAXT)
 rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ planes, PlaneDesc pd,
                const WT *__restrict__ gain, float eps, WT *__restrict__ out, WT *__restrict__ out_lo,
-               float *__restrict__ out_f32, int d, WeightPrefetch pf)
+               float *__restrict__ out_f32, int d)
 {
-    pdl_trigger();
-    prefetch_weights(pf, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
-    pdl_wait();
+    pdl_enter();
     __shared__ float red[32];
     const int t = blockIdx.x;
     float *xr = x + (size_t)t * d;
@@ -179,27 +176,25 @@ rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ planes, PlaneDes
 
 template <typename WT, int GROUPS, int MAXT>
 static void launch_rmsnorm_as(float *x, const float *planes, const PlaneDesc &pd, const void *gain, float eps, void *out,
-                              void *out_lo, float *out_f32, int T, int d, cudaStream_t s, const WeightPrefetch &pf)
+                              void *out_lo, float *out_f32, int T, int d, cudaStream_t s)
 {
     int threads = ((d / (4 * GROUPS) + 31) / 32) * 32;
     if (threads > MAXT) threads = MAXT;
     launch_pdl(rmsnorm_kernel<WT, GROUPS, MAXT>, dim3(T), dim3(threads), 0, s, x, planes, pd, (const WT *)gain, eps,
-               (WT *)out, (WT *)out_lo, out_f32, d, pf);
+               (WT *)out, (WT *)out_lo, out_f32, d);
 }
 
 void launch_add_rmsnorm(int dtype, float *x, const float *planes, const PlaneDesc &pd, const void *gain,
-                        float eps, void *out, void *out_lo, float *out_f32, int T, int d, cudaStream_t s,
-                        const WeightPrefetch *prefetch)
+                        float eps, void *out, void *out_lo, float *out_f32, int T, int d, cudaStream_t s)
 {
-    const WeightPrefetch pf = prefetch ? *prefetch : WeightPrefetch{};
     // rows of up to 4096 columns: one column group per thread; wider rows: two groups per thread in blocks of at
     // most 768 threads, which leaves the compiler 80 registers for both groups' loads in flight
     if (dtype == MEDUSA_BF16) {
-        if (d <= 4096) launch_rmsnorm_as<bf16, 1, 1024>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s, pf);
-        else launch_rmsnorm_as<bf16, 2, 768>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s, pf);
+        if (d <= 4096) launch_rmsnorm_as<bf16, 1, 1024>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s);
+        else launch_rmsnorm_as<bf16, 2, 768>(x, planes, pd, gain, eps, out, out_lo, out_f32, T, d, s);
     } else {
-        if (d <= 4096) launch_rmsnorm_as<float, 1, 1024>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s, pf);
-        else launch_rmsnorm_as<float, 2, 768>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s, pf);
+        if (d <= 4096) launch_rmsnorm_as<float, 1, 1024>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s);
+        else launch_rmsnorm_as<float, 2, 768>(x, planes, pd, gain, eps, out, nullptr, out_f32, T, d, s);
     }
 }
 
@@ -424,12 +419,9 @@ void launch_rope_apply(int dtype, const void *in, const float2 *cs, void *out, i
 template <typename AT>
 __global__ void __launch_bounds__(256)
 silu_mul_kernel(const float *__restrict__ gu, PlaneDesc pd, AT *__restrict__ act, AT *__restrict__ act_lo,
-                int F, WeightPrefetch pf)
+                int F)
 {
-    pdl_trigger();
-    prefetch_weights(pf, ((long long)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x,
-                     (long long)gridDim.x * gridDim.y * blockDim.x);
-    pdl_wait();
+    pdl_enter();
     const int t = blockIdx.y;
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= F)
@@ -455,14 +447,13 @@ silu_mul_kernel(const float *__restrict__ gu, PlaneDesc pd, AT *__restrict__ act
 }
 
 void launch_silu_mul(int dtype, const float *gate_up, const PlaneDesc &pd, void *act, void *act_lo, int T,
-                     int F, cudaStream_t s, const WeightPrefetch *prefetch)
+                     int F, cudaStream_t s)
 {
-    const WeightPrefetch pf = prefetch ? *prefetch : WeightPrefetch{};
     dim3 grid((F / 4 + 255) / 256, T);
     if (dtype == MEDUSA_BF16)
-        launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, s, gate_up, pd, (bf16 *)act, (bf16 *)act_lo, F, pf);
+        launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, s, gate_up, pd, (bf16 *)act, (bf16 *)act_lo, F);
     else
-        launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, s, gate_up, pd, (float *)act, (float *)nullptr, F, pf);
+        launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, s, gate_up, pd, (float *)act, (float *)nullptr, F);
 }
 
 // ---------------------------------------------------------------------------------------- small helpers

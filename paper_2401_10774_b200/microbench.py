@@ -35,7 +35,6 @@ def main():
     ap.add_argument("--typical", action="store_true", help="typical acceptance (0.7 / 0.09 / 0.3) instead of greedy")
     ap.add_argument("--attention", type=int, default=0, metavar="L", help="time tree_attention alone at cache length L")
     ap.add_argument("--caches", type=int, default=32)
-    ap.add_argument("--weight-prefetch", type=int, default=None, metavar="TILES")
     ap.add_argument("--device-weights", action="store_true",
                     help="draw the weights on the device (N(0, 0.02^2), not the seeded host recipe): seconds instead of a "
                          "minute of set-up, for timing runs whose numbers do not depend on the values")
@@ -45,7 +44,8 @@ def main():
 
     cfg = I.model_shape(args.model, n_layers=args.layers)
     tree_name = args.tree or ("sparse64_d5" if cfg["n_medusa"] >= 5 else "sparse64_d4")
-    spec = I.TREE_SPECS[tree_name]
+    spec = I.LARGE_TREE_SPECS[tree_name] if tree_name in I.LARGE_TREE_SPECS else I.TREE_SPECS[tree_name]
+    cfg["max_tree_nodes"] = spec["n_nodes"]
     if args.device_weights:
         gen = torch.Generator(device="cuda").manual_seed(40)
 
@@ -70,8 +70,6 @@ def main():
         dw["layers"] = [{k: dev(v) for k, v in lw.items()} for lw in w["layers"]]
     ctx = B.Context(cfg, B.BF16, args.L_max)
     ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
-    if args.weight_prefetch is not None:
-        ctx.set_option(B.OPT_WEIGHT_PREFETCH, args.weight_prefetch)
     ctx.load_weights(dw)
     # a cache of the requested length without paying for a long prefill: prefill 64 tokens, then tell the
     # library the rest is there (the K/V values beyond are zeros, which is fine for timing)
