@@ -57,6 +57,9 @@ typedef struct {
     int32_t max_tree_nodes; /* largest tree (nodes incl. root) the context must hold; 0 = 64.  Up to 256 (paper Sec. 3.3.1 /
                              * Fig. 4 studies trees of that size): buffers are sized for ceil(max/64) tiles of 64 token
                              * rows, projections and attention then run tile by tile */
+    int32_t max_batch;      /* sequences the context holds (batch > 1: paper Sec. 4 leaves batching to the serving layer; App. G
+                             * studies the operators at batch 16); 0 = 1, at most 4.  Every sequence has its own KV cache,
+                             * cache length, root token and last hidden state */
 } medusa_model_desc;
 
 /* Static tree buffers (paper Sec. 2.1.2, Fig. 2).  Host arrays owned by the caller:
@@ -138,7 +141,8 @@ enum {
 /* Creates a context on CUDA device `device`; `stream` is a cudaStream_t.  With NULL the context creates a
  * blocking stream of its own (the legacy default stream cannot be captured into the whole-step graphs); like
  * every blocking stream it orders itself with work on the legacy default stream in both directions.
- * Shapes supported: head_dim in {64,128}, T <= max_tree_nodes <= 256, d and ffn multiples of 8 (bf16) / 4 (f32). */
+ * Shapes supported: head_dim in {64,128}, T <= max_tree_nodes <= 256, max_batch <= 4, d and ffn multiples of 8 (bf16) /
+ * 4 (f32). */
 int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc, int32_t device, void *stream);
 int32_t medusa_destroy(medusa_ctx *ctx);
 const char *medusa_last_error(const medusa_ctx *ctx);
@@ -283,7 +287,7 @@ int32_t medusa_accept_and_update_kv(medusa_ctx *ctx, const void *tree_k, const v
 
 /* Registers the weights (pointers must outlive the context) and allocates the KV cache and decode state. */
 int32_t medusa_load_weights(medusa_ctx *ctx, const medusa_weights *w);
-/* Clears the decode state: cache_len = 0, status = OK. */
+/* Clears the decode state of every sequence: cache_len = 0, status = OK. */
 int32_t medusa_reset(medusa_ctx *ctx);
 /* Runs the prompt (device int32 [n]) through the backbone in chains of up to 64 tokens (a chain tree is
  * ordinary causal attention), commits every position, and leaves root = argmax of the last logits and
@@ -306,6 +310,21 @@ int32_t medusa_tree_pass(medusa_ctx *ctx, const int32_t *tokens);
  * from a buffer of the context, into which gumbel is copied first. */
 int32_t medusa_decode_step(medusa_ctx *ctx, const medusa_accept_params *params, const float *gumbel,
                            int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host);
+/* Batch > 1.  A context created with max_batch = B holds B independent sequences.  medusa_select_sequence chooses the
+ * sequence that the single-sequence calls (medusa_prefill, medusa_decode_step, medusa_tree_pass, medusa_generate and the
+ * per-sequence workspace views STATE, K_CACHE, V_CACHE, H_LAST, HEAD_LOGITS, TOPK_IDX, ACC_NODES, EMITTED) work on;
+ * medusa_reset clears all sequences.  Errors: INVALID_ARG (b outside [0, B)). */
+int32_t medusa_select_sequence(medusa_ctx *ctx, int32_t b);
+/* One decode step of ALL B sequences in one backbone pass: sequence b's tree tokens are rows 64 b .. 64 b + T - 1 of the
+ * pass (LOGITS, HIDDEN, TREE_K/V, TREE_TOK use the same rows), the projections stream the weights once for all sequences,
+ * the attention runs per sequence against that sequence's cache and cache length, and heads, top-k, acceptance and
+ * commit run per sequence exactly as in medusa_decode_step (same acceptance rule for all).  The uploaded tree must have
+ * at most 64 nodes (SHAPE otherwise).  gumbel (nullable): float [B][V] device noise rows; emitted_host [B][depth+1] and
+ * n_emitted_host [B] (nullable, pinned host memory recommended): async copies, valid after the stream is synchronised.
+ * Every sequence must have been prefilled.  The step is enqueued directly (no whole-step graph). */
+int32_t medusa_decode_step_batch(medusa_ctx *ctx, const medusa_accept_params *params, const float *gumbel,
+                                 int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host);
+
 /* Convenience loop with HOST buffers: prefill prompt_host[n_prompt], then decode steps until G tokens are
  * emitted (one stream synchronisation per step to read the emitted tokens).  gumbel_host (nullable):
  * [max steps = G][V].  Writes out_tokens_host[G]; emitted_per_step_host (nullable) [G]; *steps_host. */

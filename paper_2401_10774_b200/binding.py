@@ -34,7 +34,7 @@ class ModelDesc(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("ffn", C.c_int32), ("vocab", C.c_int32), ("n_medusa", C.c_int32), ("dtype", C.c_int32),
                 ("L_max", C.c_int32), ("n_kv_heads", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float),
-                ("max_tree_nodes", C.c_int32)]
+                ("max_tree_nodes", C.c_int32), ("max_batch", C.c_int32)]
 
 
 class TreeBuffers(C.Structure):
@@ -144,7 +144,7 @@ class Context:
         desc = ModelDesc(n_layers=cfg["n_layers"], d=cfg["d"], n_heads=cfg["n_heads"], head_dim=cfg["head_dim"],
                          ffn=cfg["ffn"], vocab=cfg["vocab"], n_medusa=cfg["n_medusa"], dtype=dtype, L_max=L_max,
                          n_kv_heads=cfg.get("n_kv_heads", 0), rms_eps=cfg.get("rms_eps", 1e-5), rope_theta=cfg.get("rope_theta", 1e4),
-                         max_tree_nodes=cfg.get("max_tree_nodes", 0))
+                         max_tree_nodes=cfg.get("max_tree_nodes", 0), max_batch=cfg.get("max_batch", 0))
         self.handle = C.c_void_p(0)
         sp = C.c_void_p(0 if stream is None else int(stream))
         rc = lib().medusa_create(C.byref(self.handle), C.byref(desc), C.c_int32(device), sp)
@@ -226,6 +226,13 @@ class Context:
     def decode_step(self, params: AcceptParams, gumbel=None, max_commit=1 << 30, emitted_host=None, n_emitted_host=None):
         self._check(lib().medusa_decode_step(self.handle, C.byref(params), _ptr(gumbel), C.c_int32(int(max_commit)),
                                              _ptr(emitted_host), _ptr(n_emitted_host)))
+
+    def select_sequence(self, b: int):
+        self._check(lib().medusa_select_sequence(self.handle, C.c_int32(int(b))))
+
+    def decode_step_batch(self, params: AcceptParams, gumbel=None, max_commit=1 << 30, emitted_host=None, n_emitted_host=None):
+        self._check(lib().medusa_decode_step_batch(self.handle, C.byref(params), _ptr(gumbel), C.c_int32(int(max_commit)),
+                                                   _ptr(emitted_host), _ptr(n_emitted_host)))
 
     def generate(self, prompt_host: np.ndarray, G: int, params: AcceptParams, gumbel_host=None) -> dict:
         prompt = np.ascontiguousarray(prompt_host, dtype=np.int32)

@@ -21,7 +21,17 @@ using namespace medusa;
 struct medusa_ctx {
     medusa_model_desc m{};
     int device = 0;
-    int rows = TREE_ROWS;  // token rows the context's buffers hold: 64 * ceil(max_tree_nodes / 64), at most MAX_T
+    int rows = TREE_ROWS;  // token rows the context's buffers hold: 64 * max(ceil(max_tree_nodes / 64), max_batch), at most MAX_T
+    // Sequences (batch): every sequence has its own decode state, KV cache, last hidden state and per-step integer
+    // outputs.  The members d_state, k_cache, v_cache, h_last, head_x, head_logits, topk_idx, acc_nodes, emitted,
+    // gumbel_dev and L_upper below are VIEWS of the selected sequence `cur` into the *_all allocations
+    // (medusa_select_sequence re-points them), so that every single-sequence call works on the selected sequence.
+    int B = 1, cur = 0;
+    int32_t *state_all = nullptr, *topk_idx_all = nullptr, *acc_nodes_all = nullptr, *emitted_all = nullptr;
+    float *h_last_all = nullptr, *head_x_all = nullptr, *head_logits_all = nullptr, *gumbel_all = nullptr;
+    char *k_cache_all = nullptr, *v_cache_all = nullptr;
+    size_t cache_seq_bytes = 0;  // bytes of one sequence's K (or V) cache
+    std::vector<int> L_upper_all;
     int Hkv = 0;  // key/value heads: m.n_kv_heads, or m.n_heads when that is 0 (ordinary multi-head attention)
     cudaStream_t stream = nullptr;
     bool own_stream = false;
@@ -97,7 +107,7 @@ struct medusa_ctx {
     // the values in StepKey (the cache length is read on the device); the second consecutive step with the same key is captured from the stream into an
     // executable graph, and later steps with that key replay it.  MEDUSA_STEP_GRAPH=0 turns this off.
     struct StepKey {
-        int32_t max_commit, has_gumbel;
+        int32_t max_commit, has_gumbel, seq;
         medusa_accept_params p;
         int32_t *emitted_host, *n_emitted_host;
     };
@@ -296,16 +306,27 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
 
 // One backbone pass over T token rows (paper App. G Table 5, "parallel decoding" column).
 // logits are produced for rows [lm_row0, T).
-int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *mask, const int32_t *pos, int lm_row0,
-                  int mask_words)
+// n_seq == 1: the T tokens of the selected sequence occupy rows 0..T-1.  n_seq > 1 (a batched step): sequence b's T_seq
+// tree tokens occupy rows 64 b .. 64 b + T_seq - 1 of every buffer; the row-wise kernels and the projections run over
+// all 64 n_seq rows at once (the weights are streamed once for all sequences), the rotary table and the attention run
+// per sequence against that sequence's own cache and cache length.
+int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_t *mask, const int32_t *pos, int lm_row0,
+                  int mask_words, int n_seq = 1)
 {
     const medusa_model_desc &m = c->m;
     const int d = m.d, H = m.n_heads, Hkv = c->Hkv, D = m.head_dim, HD = H * D, HkvD = Hkv * D, F = m.ffn, dt = m.dtype;
     const int qkv_ld = HD + 2 * HkvD;  // a row of the QKV projection: [q | k | v]
     cudaStream_t s = c->stream;
+    const int T = n_seq > 1 ? n_seq * TREE_ROWS : T_seq;  // rows of the pass
     int32_t *cache_len = c->d_state + ST_CACHE_LEN;
     PROF(c, PC_ELEMWISE, 1, launch_embed(dt, tokens, c->w.embed, c->x, T, d, m.vocab, s));
-    PROF(c, PC_ELEMWISE, 1, launch_rope_table(c->rope_cs, cache_len, pos, T, D, m.rope_theta, s));
+    if (n_seq > 1) {
+        for (int b = 0; b < n_seq; ++b)
+            PROF(c, PC_ELEMWISE, 1, launch_rope_table(c->rope_cs + (size_t)b * TREE_ROWS * (D / 2), c->state_all + (size_t)b * ST_WORDS + ST_CACHE_LEN,
+                                                      pos, T_seq, D, m.rope_theta, s));
+    } else {
+        PROF(c, PC_ELEMWISE, 1, launch_rope_table(c->rope_cs, cache_len, pos, T, D, m.rope_theta, s));
+    }
     MEDUSA_LAUNCH_CHECK(c);
     PlaneDesc pd_prev{};  // planes of the previous projection still to be added to the residual stream
     for (int l = 0; l < m.n_layers; ++l) {
@@ -343,8 +364,24 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T, const uint64_t *m
             PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd_kv, HD, c->rope_cs, c->q, c->lo(c->q, HD), tk, tv, T, H, Hkv, D, s));
         }
         MEDUSA_LAUNCH_CHECK(c);
-        TRY(attention(c, c->q, tk, tv, kc, vc, cache_len, mask, c->att, c->lo(c->att, HD), nullptr, T, c->L_upper, true,
-                      mask_words, c->lo(c->q, HD)));
+        if (n_seq > 1) {
+            // every sequence's 64-row tile against its own cache (launches follow one another on the stream and each
+            // waits for its predecessor before it touches anything, so they can share the split-KV workspace)
+            for (int b = 0; b < n_seq; ++b) {
+                const size_t ro = (size_t)b * TREE_ROWS;  // first row of the sequence
+                const size_t lay = (size_t)l * Hkv * m.L_max * D * c->esz;
+                const char *q_lo = (const char *)c->lo(c->q, HD);
+                char *att_lo = (char *)c->lo(c->att, HD);
+                TRY(attention(c, (const char *)c->q + ro * HD * c->esz, tk + ro * HkvD * c->esz, tv + ro * HkvD * c->esz,
+                              c->k_cache_all + (size_t)b * c->cache_seq_bytes + lay, c->v_cache_all + (size_t)b * c->cache_seq_bytes + lay,
+                              c->state_all + (size_t)b * ST_WORDS + ST_CACHE_LEN, mask, (char *)c->att + ro * HD * c->esz,
+                              att_lo ? att_lo + ro * HD * c->esz : nullptr, nullptr, T_seq, c->L_upper_all[b], true, mask_words,
+                              q_lo ? q_lo + ro * HD * c->esz : nullptr));
+            }
+        } else {
+            TRY(attention(c, c->q, tk, tv, kc, vc, cache_len, mask, c->att, c->lo(c->att, HD), nullptr, T, c->L_upper, true,
+                          mask_words, c->lo(c->q, HD)));
+        }
         if (l == c->tap_layer)
             MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_att, c->att, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)c->rows * HD * c->esz,
                                            cudaMemcpyDeviceToDevice, s));
@@ -389,6 +426,25 @@ int32_t check_ready(medusa_ctx *c, bool need_tree, bool need_weights)
 
 static void drop_step_graphs(medusa_ctx *c);
 
+// Re-points the selected-sequence views at sequence b (host pointer arithmetic only).
+static void point_at(medusa_ctx *c, int b)
+{
+    const medusa_model_desc &m = c->m;
+    const size_t K = m.n_medusa ? m.n_medusa : 1, R = (size_t)c->rows;
+    c->cur = b;
+    c->d_state = c->state_all + (size_t)b * ST_WORDS;
+    c->h_last = c->h_last_all + (size_t)b * m.d;
+    c->head_x = c->head_x_all + (size_t)b * K * m.d;
+    c->head_logits = c->head_logits_all + (size_t)b * K * m.vocab;
+    c->topk_idx = c->topk_idx_all + (size_t)b * K * R;
+    c->acc_nodes = c->acc_nodes_all + (size_t)b * TREE_ROWS;
+    c->emitted = c->emitted_all + (size_t)b * TREE_ROWS;
+    c->gumbel_dev = c->gumbel_all + (size_t)b * m.vocab;
+    c->k_cache = c->k_cache_all ? c->k_cache_all + (size_t)b * c->cache_seq_bytes : nullptr;
+    c->v_cache = c->v_cache_all ? c->v_cache_all + (size_t)b * c->cache_seq_bytes : nullptr;
+    if ((size_t)b < c->L_upper_all.size()) c->L_upper = c->L_upper_all[b];
+}
+
 extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc, int32_t device, void *stream)
 {
     if (!out || !desc) return MEDUSA_ERR_INVALID_ARG;
@@ -399,6 +455,8 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
         return MEDUSA_ERR_INVALID_ARG;
     if (m.max_tree_nodes < 0 || m.max_tree_nodes > MAX_T)
         return MEDUSA_ERR_SHAPE;  // trees of up to MAX_T nodes
+    if (m.max_batch < 0 || m.max_batch > MAX_T / TREE_ROWS)
+        return MEDUSA_ERR_SHAPE;  // up to MAX_T / 64 sequences (one tile of 64 token rows each)
     if (m.n_kv_heads < 0 || (m.n_kv_heads > 0 && m.n_heads % m.n_kv_heads != 0))
         return MEDUSA_ERR_SHAPE;  // every key/value head serves the same number of query heads
     const int vn = m.dtype == MEDUSA_BF16 ? 8 : 4;
@@ -414,6 +472,9 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     c->m = m;
     c->device = device;
     c->rows = m.max_tree_nodes <= TREE_ROWS ? TREE_ROWS : ((m.max_tree_nodes + TREE_ROWS - 1) / TREE_ROWS) * TREE_ROWS;
+    c->B = m.max_batch > 1 ? m.max_batch : 1;
+    if (c->rows < c->B * TREE_ROWS) c->rows = c->B * TREE_ROWS;  // a batched pass gives every sequence one tile of 64 rows
+    c->L_upper_all.assign(c->B, 0);
     c->stream = (cudaStream_t)stream;
     if (!c->stream) {
         // The legacy default stream cannot be captured into a graph.  A blocking stream orders itself with the
@@ -430,7 +491,8 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     c->Hkv = m.n_kv_heads > 0 ? m.n_kv_heads : m.n_heads;
     const size_t d = m.d, HD = (size_t)m.n_heads * m.head_dim, HkvD = (size_t)c->Hkv * m.head_dim, F = m.ffn, V = m.vocab,
                  K = m.n_medusa, R = (size_t)c->rows;
-    TRY(dev_alloc(c, &c->d_state, ST_WORDS));
+    const size_t NB = (size_t)c->B;
+    TRY(dev_alloc(c, &c->state_all, NB * ST_WORDS));
     TRY(dev_alloc(c, &c->d_mask, R * (R / 64)));
     TRY(dev_alloc(c, &c->d_chain_mask, R));
     TRY(dev_alloc(c, &c->d_pos, R));
@@ -447,22 +509,23 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     TRY(dev_alloc(c, &c->hidden_f32, R * d));
     TRY(dev_alloc_bytes(c, &c->act, planes * R * F * c->esz));
     TRY(dev_alloc_bytes(c, &c->hidden, planes * R * d * c->esz));
-    TRY(dev_alloc(c, &c->h_last, d));
-    TRY(dev_alloc(c, &c->head_x, (K ? K : 1) * d));
+    TRY(dev_alloc(c, &c->h_last_all, NB * d));
+    TRY(dev_alloc(c, &c->head_x_all, NB * (K ? K : 1) * d));
     TRY(dev_alloc(c, &c->logits, R * V));
-    TRY(dev_alloc(c, &c->head_logits, (K ? K : 1) * V));
+    TRY(dev_alloc(c, &c->head_logits_all, NB * (K ? K : 1) * V));
     TRY(dev_alloc(c, &c->rope_cs, R * (size_t)(m.head_dim / 2)));
-    TRY(dev_alloc(c, &c->topk_idx, (K ? K : 1) * R));
+    TRY(dev_alloc(c, &c->topk_idx_all, NB * (K ? K : 1) * R));
     TRY(dev_alloc(c, &c->tree_tok, R));
-    TRY(dev_alloc(c, &c->acc_nodes, R));
-    TRY(dev_alloc(c, &c->emitted, R));
+    TRY(dev_alloc(c, &c->acc_nodes_all, NB * TREE_ROWS));
+    TRY(dev_alloc(c, &c->emitted_all, NB * TREE_ROWS));
     TRY(dev_alloc(c, &c->node_argmax, R));
     TRY(dev_alloc(c, &c->iota, R));
-    TRY(dev_alloc(c, &c->tmp_i32, 8));
+    TRY(dev_alloc(c, &c->tmp_i32, 8 * NB));
     TRY(dev_alloc(c, &c->node_lse, R));
     TRY(dev_alloc(c, &c->node_ent, R));
     TRY(dev_alloc_bytes(c, &c->node_part, R * NODE_STAT_SLICES * NODE_PART_BYTES));
-    TRY(dev_alloc(c, &c->gumbel_dev, V));
+    TRY(dev_alloc(c, &c->gumbel_all, NB * V));
+    point_at(c, 0);
     TRY(dev_alloc_bytes(c, &c->topk_scratch, topk_scratch_bytes(m.n_medusa > 0 ? m.n_medusa : 1)));
     TRY(dev_alloc(c, &c->tap_x_in, R * d));
     TRY(dev_alloc(c, &c->tap_x_out, R * d));
@@ -557,7 +620,7 @@ static const void *workspace_view(medusa_ctx *c, int32_t which, size_t *bytes)
     const medusa_model_desc &m = c->m;
     const size_t R = (size_t)c->rows, d = m.d, V = m.vocab, K = m.n_medusa ? m.n_medusa : 1, HD = (size_t)m.n_heads * m.head_dim;
     const size_t HkvD = (size_t)c->Hkv * m.head_dim, planes = m.dtype == MEDUSA_BF16 ? 2 : 1;
-    const size_t cache_bytes = (size_t)m.n_layers * HkvD * m.L_max * c->esz, tree_bytes = (size_t)m.n_layers * R * HkvD * c->esz;
+    const size_t cache_bytes = c->cache_seq_bytes, tree_bytes = (size_t)m.n_layers * R * HkvD * c->esz;
     const void *p = nullptr;
     size_t n = 0;
     switch (which) {
@@ -570,10 +633,10 @@ static const void *workspace_view(medusa_ctx *c, int32_t which, size_t *bytes)
     case MEDUSA_WS_HEAD_LOGITS: p = c->head_logits; n = K * V * sizeof(float); break;
     case MEDUSA_WS_TOPK_IDX: p = c->topk_idx; n = K * R * sizeof(int32_t); break;
     case MEDUSA_WS_TREE_TOK: p = c->tree_tok; n = R * sizeof(int32_t); break;
-    case MEDUSA_WS_ACC_NODES: p = c->acc_nodes; n = R * sizeof(int32_t); break;
+    case MEDUSA_WS_ACC_NODES: p = c->acc_nodes; n = TREE_ROWS * sizeof(int32_t); break;
     case MEDUSA_WS_STATE: p = c->d_state; n = ST_WORDS * sizeof(int32_t); break;
     case MEDUSA_WS_H_LAST: p = c->h_last; n = d * sizeof(float); break;
-    case MEDUSA_WS_EMITTED: p = c->emitted; n = R * sizeof(int32_t); break;
+    case MEDUSA_WS_EMITTED: p = c->emitted; n = TREE_ROWS * sizeof(int32_t); break;
     case MEDUSA_WS_TAP_X_IN: p = c->tap_x_in; n = R * d * sizeof(float); break;
     case MEDUSA_WS_TAP_X_OUT: p = c->tap_x_out; n = R * d * sizeof(float); break;
     case MEDUSA_WS_TAP_ATT: p = c->tap_att; n = planes * R * HD * c->esz; break;
@@ -869,12 +932,14 @@ extern "C" int32_t medusa_load_weights(medusa_ctx *c, const medusa_weights *w)
     c->w = *w;
     c->w.layers_host = nullptr;
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
-    if (!c->k_cache) {
+    if (!c->k_cache_all) {
         const size_t HkvD = (size_t)c->Hkv * m.head_dim;
         const size_t cache_bytes = (size_t)m.n_layers * HkvD * m.L_max * c->esz;
         const size_t tree_bytes = (size_t)m.n_layers * c->rows * HkvD * c->esz;
-        TRY(dev_alloc_bytes(c, &c->k_cache, cache_bytes));
-        TRY(dev_alloc_bytes(c, &c->v_cache, cache_bytes));
+        c->cache_seq_bytes = cache_bytes;
+        TRY(dev_alloc_bytes(c, (void **)&c->k_cache_all, cache_bytes * c->B));
+        TRY(dev_alloc_bytes(c, (void **)&c->v_cache_all, cache_bytes * c->B));
+        point_at(c, c->cur);
         TRY(dev_alloc_bytes(c, &c->tree_k, tree_bytes));
         TRY(dev_alloc_bytes(c, &c->tree_v, tree_bytes));
     }
@@ -900,7 +965,8 @@ extern "C" int32_t medusa_reset(medusa_ctx *c)
 {
     if (!c) return MEDUSA_ERR_INVALID_ARG;
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
-    MEDUSA_CUDA(c, cudaMemsetAsync(c->d_state, 0, ST_WORDS * sizeof(int32_t), c->stream));
+    MEDUSA_CUDA(c, cudaMemsetAsync(c->state_all, 0, (size_t)c->B * ST_WORDS * sizeof(int32_t), c->stream));
+    c->L_upper_all.assign(c->B, 0);
     c->L_upper = 0;
     return MEDUSA_OK;
 }
@@ -1059,6 +1125,7 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
         medusa_ctx::StepKey key;
         memset(&key, 0, sizeof key);
         key.max_commit = max_commit;
+        key.seq = c->cur;
         const bool noisy = gumbel && params->mode == MEDUSA_TYPICAL;  // the acceptance kernel's own condition
         key.has_gumbel = noisy ? 1 : 0;
         key.p = *params;
@@ -1088,6 +1155,77 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
     c->L_upper += max_commit;
     if (c->L_upper > m.L_max) c->L_upper = m.L_max;
     return MEDUSA_OK;
+}
+
+extern "C" int32_t medusa_select_sequence(medusa_ctx *c, int32_t b)
+{
+    if (!c) return MEDUSA_ERR_INVALID_ARG;
+    if (b < 0 || b >= c->B) return fail(c, MEDUSA_ERR_INVALID_ARG, "sequence %d: the context holds %d sequence(s)", b, c->B);
+    c->L_upper_all[c->cur] = c->L_upper;
+    point_at(c, b);
+    c->have_last_key = false;  // the next step belongs to another sequence: its graph is found by the key's sequence index
+    return MEDUSA_OK;
+}
+
+// One step of ALL sequences of the context in one backbone pass (batch > 1): the heads and the integer stages run per
+// sequence, the projections once over all sequences' token rows.
+extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_params *params, const float *gumbel,
+                                            int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host)
+{
+    TRY(check_ready(c, true, true));
+    if (!params) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: null params");
+    if (max_commit < 1) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: max_commit must be >= 1");
+    if (params->mode != MEDUSA_GREEDY && params->mode != MEDUSA_TYPICAL)
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: unknown mode %d", params->mode);
+    if (c->tree.T > TREE_ROWS)
+        return fail(c, MEDUSA_ERR_SHAPE, "a batched step gives every sequence one tile of 64 token rows: the tree has %d nodes", c->tree.T);
+    const medusa_model_desc &m = c->m;
+    const int B = c->B, depth1 = c->tree.depth + 1, T = c->tree.T;
+    if (max_commit > depth1) max_commit = depth1;
+    MEDUSA_CUDA(c, cudaSetDevice(c->device));
+    const int keep = c->cur;
+    c->L_upper_all[keep] = c->L_upper;
+    int32_t rc = MEDUSA_OK;
+    // (1) candidates of every sequence: heads on its last accepted hidden state, top-k, its tile of tree tokens
+    for (int b = 0; b < B && rc == MEDUSA_OK; ++b) {
+        point_at(c, b);
+        rc = heads_impl(c, c->h_last, 1, c->w.medusa_w1, c->w.medusa_w2, c->d_state + ST_ROOT, c->topk_idx, nullptr, nullptr,
+                        c->tree_tok + (size_t)b * TREE_ROWS);
+    }
+    // (2) one backbone pass over all sequences' tiles
+    if (rc == MEDUSA_OK) rc = tree_pass(c, c->tree_tok, T, c->d_mask, c->d_pos, 0, c->tree.mask_words, B);
+    // (3) acceptance and commit, sequence by sequence
+    for (int b = 0; b < B && rc == MEDUSA_OK; ++b) {
+        point_at(c, b);
+        int32_t *st = c->d_state;
+        const size_t ro = (size_t)b * TREE_ROWS;
+        rc = medusa_evaluate_posterior(c, c->logits + ro * m.vocab, c->tree_tok + ro, params,
+                                       gumbel ? gumbel + (size_t)b * m.vocab : nullptr, st + ST_BEST, st + ST_ACCEPT_LEN,
+                                       st + ST_NEXT_ROOT, c->acc_nodes);
+        if (rc != MEDUSA_OK) break;
+        CommitArgs a{};
+        const size_t HkvD = (size_t)c->Hkv * m.head_dim;
+        a.tree_k = (const char *)c->tree_k + ro * HkvD * c->esz; a.tree_v = (const char *)c->tree_v + ro * HkvD * c->esz;
+        a.k_cache = c->k_cache; a.v_cache = c->v_cache;
+        a.acc_nodes = c->acc_nodes; a.accept_len = st + ST_ACCEPT_LEN; a.max_commit = max_commit;
+        a.cache_len = st + ST_CACHE_LEN; a.hidden = c->hidden_f32 + ro * m.d; a.h_last = c->h_last; a.tree_tok = c->tree_tok + ro;
+        a.emitted = c->emitted; a.n_emitted = st + ST_N_EMITTED; a.status = st + ST_STATUS;
+        a.next_root = st + ST_NEXT_ROOT; a.root_out = st + ST_ROOT;
+        a.tree_rows = c->rows; a.n_layers = m.n_layers; a.H = c->Hkv; a.D = m.head_dim; a.L_max = m.L_max; a.d = m.d;
+        a.depth_plus1 = depth1;
+        PROF(c, PC_COMMIT, 2, launch_commit(m.dtype, a, c->stream));
+        if (cudaGetLastError() != cudaSuccess) { rc = fail(c, MEDUSA_ERR_CUDA, "commit launch failed"); break; }
+        if (emitted_host &&
+            cudaMemcpyAsync(emitted_host + (size_t)b * depth1, c->emitted, depth1 * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+            rc = fail(c, MEDUSA_ERR_CUDA, "copy of the emitted tokens failed");
+        if (n_emitted_host &&
+            cudaMemcpyAsync(n_emitted_host + b, st + ST_N_EMITTED, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+            rc = fail(c, MEDUSA_ERR_CUDA, "copy of the emitted count failed");
+        int up = c->L_upper_all[b] + max_commit;
+        c->L_upper_all[b] = up > m.L_max ? m.L_max : up;
+    }
+    point_at(c, keep);
+    return rc;
 }
 
 extern "C" int32_t medusa_generate(medusa_ctx *c, const int32_t *prompt_host, int32_t n_prompt, int32_t G,
