@@ -54,6 +54,10 @@ WORKLOADS = {
     "7b_tree256": dict(name="7b_medusa1_greedy_step_tree256", model="7b", tree="sparse256_d4", prompt=512, L_max=4096,
                        weights_seed=40, prompt_seed=41, mode="greedy", oracle_layers=1,
                        metric="decode tokens/s (7B-shape bf16 Medusa tree-verification step, 256-node tree, batch 1)"),
+    # batch > 1: four sequences (own caches, prompts of 512 tokens from four seeds) stepped in one backbone pass
+    "7b_batch4": dict(name="7b_medusa1_greedy_step_batch4", model="7b", tree="sparse64_d4", prompt=512, L_max=4096,
+                      weights_seed=40, prompt_seed=41, mode="greedy", oracle_layers=2, batch=4,
+                      metric="decode tokens/s, all sequences (7B-shape bf16 Medusa tree-verification step, 64-node tree, batch 4)"),
     "13b": dict(name="13b_medusa_typical_step", model="13b", tree="sparse64_d5", prompt=3584, L_max=4096, weights_seed=50,
                 prompt_seed=51, noise_seed=52, mode="typical", temperature=0.7, eps=0.09, delta=0.3, oracle_layers=4,
                 metric="decode tokens/s (13B-shape bf16 Medusa tree-verification step, 64-node depth-5 tree, typical "
@@ -260,7 +264,8 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     spec = tree_spec(WORKLOAD["tree"])
-    cfg = I.model_shape(WORKLOAD["model"], max_tree_nodes=spec["n_nodes"])
+    NB = int(WORKLOAD.get("batch", 1))  # sequences stepped together
+    cfg = I.model_shape(WORKLOAD["model"], max_tree_nodes=spec["n_nodes"], max_batch=NB)
     t_setup = time.perf_counter()
     w = I.make_weights(cfg, seed=WORKLOAD["weights_seed"], dtype="bf16")
 
@@ -277,9 +282,20 @@ def run_gpu(args):
     ctx = B.Context(cfg, B.BF16, WORKLOAD["L_max"], device=local, stream=stream.cuda_stream)
     tree = ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
     ctx.load_weights(dw)
-    prompt = I.make_prompt(WORKLOAD["prompt"], cfg["vocab"], WORKLOAD["prompt_seed"])
-    ctx.prefill(torch.from_numpy(prompt).cuda())
+    for b in range(NB):
+        ctx.select_sequence(b)
+        prompt = I.make_prompt(WORKLOAD["prompt"], cfg["vocab"], WORKLOAD["prompt_seed"] + 100 * b)
+        ctx.prefill(torch.from_numpy(prompt).cuda())
+    ctx.select_sequence(0)
     torch.cuda.synchronize()
+
+    def total_len():
+        n = 0
+        for b in range(NB):
+            ctx.select_sequence(b)
+            n += ctx.state()["cache_len"]
+        ctx.select_sequence(0)
+        return n
     t_setup = time.perf_counter() - t_setup
     typical = WORKLOAD["mode"] == "typical"
     if typical:
@@ -287,8 +303,8 @@ def run_gpu(args):
     else:
         params = B.AcceptParams(mode=B.GREEDY)
     W = tree["depth"] + 1
-    pinned = torch.zeros(W + 1, dtype=torch.int32).pin_memory()
-    emitted_ptr, n_ptr = pinned.data_ptr(), pinned.data_ptr() + 4 * W
+    pinned = torch.zeros(NB * (W + 1), dtype=torch.int32).pin_memory()
+    emitted_ptr, n_ptr = pinned.data_ptr(), pinned.data_ptr() + 4 * W * NB
     # typical acceptance samples the next root with Gumbel noise the caller supplies: one float [V] row per step
     n_prof = min(args.steps, 5)
     n_noise = 2 * args.warmup + 3 * args.steps + n_prof
@@ -302,7 +318,10 @@ def run_gpu(args):
     def step_device_only():
         i = step_no[0]
         step_no[0] += 1
-        ctx.decode_step(params, noise_dev[i] if typical else None, 1 << 30, None, None)
+        if NB > 1:
+            ctx.decode_step_batch(params, None, 1 << 30, None, None)
+        else:
+            ctx.decode_step(params, noise_dev[i] if typical else None, 1 << 30, None, None)
 
     def step_e2e():
         # what a caller does: hand the step its host-side input (the noise row, if the mode draws one), run it,
@@ -311,6 +330,10 @@ def run_gpu(args):
         step_no[0] += 1
         if typical:
             noise_stage.copy_(noise_host[i], non_blocking=True)
+        if NB > 1:
+            ctx.decode_step_batch(params, None, 1 << 30, emitted_ptr, n_ptr)
+            torch.cuda.synchronize()
+            return int(pinned[W * NB:W * NB + NB].sum())
         ctx.decode_step(params, noise_stage if typical else None, 1 << 30, emitted_ptr, n_ptr)
         torch.cuda.synchronize()
         return int(pinned[W])
@@ -321,7 +344,7 @@ def run_gpu(args):
     for _ in range(args.warmup):
         step_device_only()
     read_peak_gbs = measure_read_peak(torch, B, stream)
-    L0 = ctx.state()["cache_len"]
+    L0 = total_len()
     ctx.get_profile(reset=True)
     sampler = ClockSampler(local)
     sampler.start()
@@ -337,7 +360,7 @@ def run_gpu(args):
     ms = e0.elapsed_time(e1)
     prof = ctx.get_profile(reset=True)
     launches = sum(v["launches"] for v in prof.values())
-    L1 = ctx.state()["cache_len"]
+    L1 = total_len()
     tokens = L1 - L0
     # ---- timed region 2: the same K steps through the host-buffer call, tokens read back every step
     barrier()
@@ -367,7 +390,7 @@ def run_gpu(args):
         step_device_only()
     prof_t = ctx.get_profile(reset=True)
     ctx.set_profiling(False)
-    L_end = ctx.state()["cache_len"]
+    L_end = total_len() // NB
     status = ctx.device_status()
     if status != 0:
         raise SystemExit("device status %d during the benchmark" % status)
@@ -380,19 +403,22 @@ def run_gpu(args):
     if rank == 0:
         peaks = measured_peaks()
         T = tree["T"]
-        L_mid = (L0 + L1) // 2
+        L_mid = (L0 + L1) // (2 * NB)
         sb = R.step_bytes(dict(cfg, depth=tree["depth"]), T, L_mid, tree["depth"])
+        if NB > 1:  # the weights cross the HBM once for all sequences; caches, tree K/V and logits once per sequence
+            per_seq = sb["kv_read"] + sb["tree_kv_write"] + sb["logits_write_read"] + sb["commit"]
+            sb["total"] += (NB - 1) * per_seq
         ms_step = ms / args.steps
         step_gbs = sb["total"] / (ms_step * 1e-3) / 1e9
         # dominant kernel: the backbone GEMM launches (7 per layer + LM head)
         gemm = prof_t["gemm"]
-        gemm_bytes_step = R.gemm_launch_bytes_per_step(cfg, T)
+        gemm_bytes_step = R.gemm_launch_bytes_per_step(cfg, T * NB)
         gemm_launches_step = gemm["launches"] / max(n_prof, 1)
         gemm_ms_step = gemm["ms"] / max(n_prof, 1)
         achieved = gemm_bytes_step / (gemm_ms_step * 1e-3) / 1e9 if gemm_ms_step > 0 else 0.0
         kernels = {k: dict(ms_per_step=v["ms"] / max(n_prof, 1), launches_per_step=v["launches"] / max(n_prof, 1))
                    for k, v in prof_t.items() if v["launches"]}
-        att_bytes = cfg["n_layers"] * R.attention_bytes(T, cfg["n_heads"], cfg["head_dim"], L_end, Hkv=I.kv_heads(cfg))
+        att_bytes = NB * cfg["n_layers"] * R.attention_bytes(T, cfg["n_heads"], cfg["head_dim"], L_end, Hkv=I.kv_heads(cfg))
         if "tree_attention" in kernels and kernels["tree_attention"]["ms_per_step"] > 0:
             kernels["tree_attention"]["achieved_gbs"] = att_bytes / (kernels["tree_attention"]["ms_per_step"] * 1e-3) / 1e9
         if "heads_gemv" in kernels and kernels["heads_gemv"]["ms_per_step"] > 0:
@@ -410,19 +436,19 @@ def run_gpu(args):
             "ms_per_step": ms_step,
             "step_us": ms_step * 1e3,
             "step_us_p10_p50_p90": [float(np.percentile(per_step_us, q)) for q in (10, 50, 90)],
-            "accepted_tokens_per_step": tokens / (args.steps * world),
+            "accepted_tokens_per_step": tokens / (args.steps * world * NB),
             "higher_is_better": True,
             "scaling": "weak",
             "vs_baseline": None,
             "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": WORKLOAD["name"], "tree_nodes": T, "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"],
-                       "cache_len_start": L0, "heads": cfg["n_medusa"], "replicas": world,
+                       "cache_len_start": L0 // NB, "heads": cfg["n_medusa"], "replicas": world, "batch": NB,
                        "l2": "inputs larger than L2: every step streams %.1f GB of weights" % (sb["gemm_weights"] / 1e9)},
             "clocks": clocks,
             "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": "tokens/s",
                     "h2d_bytes_per_step": 4 * cfg["vocab"] if typical else 0,
-                    "d2h_bytes_per_step": 4 * (W + 1), "ms_per_step": ms_e2e / args.steps,
+                    "d2h_bytes_per_step": 4 * (W + 1) * NB, "ms_per_step": ms_e2e / args.steps,
                     "note": "per step: C-ABI decode_step with pinned host output buffers, stream synchronised and the "
                             "emitted tokens read on the host; " + (
                                 "the step's Gumbel noise row is copied from pinned host memory first" if typical else
@@ -449,8 +475,10 @@ def run_gpu(args):
             t0 = time.perf_counter()
             sample = OracleSample(WORKLOAD["oracle_layers"], cfg, L_mid)
             sec, desc = sample.run()
+            if NB > 1:
+                desc += "; one sequence timed, the oracle steps the %d sequences one after the other: time x %d" % (NB, NB)
             line["cpu_baseline"] = {"value": 1.0 / sec, "unit": "tokens/s", "cores": sample.cores, "kind": "oracle", "sample": desc,
-                                    "seconds_per_step": sec, "wall_s": time.perf_counter() - t0}
+                                    "seconds_per_step": sec * NB, "wall_s": time.perf_counter() - t0}
         print(json.dumps(line))
     ctx.close()
     if world > 1:

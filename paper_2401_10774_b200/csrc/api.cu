@@ -364,7 +364,16 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
             PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd_kv, HD, c->rope_cs, c->q, c->lo(c->q, HD), tk, tv, T, H, Hkv, D, s));
         }
         MEDUSA_LAUNCH_CHECK(c);
-        if (n_seq > 1) {
+        if (n_seq > 1 && c->flash_ws && c->attn_mode != 2) {
+            // all sequences in one launch of the flash kernel: grid z = sequence, each against its own cache and length
+            cudaError_t e = cudaSuccess;
+            const size_t lay = (size_t)l * Hkv * m.L_max * D * c->esz;
+            PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_flash(c->q, tk, tv, c->k_cache_all + lay, c->v_cache_all + lay,
+                                                                     c->state_all + ST_CACHE_LEN, mask, c->att, c->lo(c->att, HD), nullptr,
+                                                                     c->flash_ws, T_seq, H, Hkv, m.L_max, m.L_max, s, c->lo(c->q, HD),
+                                                                     mask_words, n_seq, (long long)(c->cache_seq_bytes / c->esz), ST_WORDS));
+            if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "batched flash attention launch failed: %s", cudaGetErrorString(e));
+        } else if (n_seq > 1) {
             // every sequence's 64-row tile against its own cache (launches follow one another on the stream and each
             // waits for its predecessor before it touches anything, so they can share the split-KV workspace)
             for (int b = 0; b < n_seq; ++b) {
@@ -1186,11 +1195,30 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
     const int keep = c->cur;
     c->L_upper_all[keep] = c->L_upper;
     int32_t rc = MEDUSA_OK;
-    // (1) candidates of every sequence: heads on its last accepted hidden state, top-k, its tile of tree tokens
-    for (int b = 0; b < B && rc == MEDUSA_OK; ++b) {
-        point_at(c, b);
-        rc = heads_impl(c, c->h_last, 1, c->w.medusa_w1, c->w.medusa_w2, c->d_state + ST_ROOT, c->topk_idx, nullptr, nullptr,
-                        c->tree_tok + (size_t)b * TREE_ROWS);
+    // (1) candidates of every sequence: the heads of all sequences in two launches (every head weight is read once),
+    // then top-k and the sequence's tile of tree tokens per sequence
+    {
+        const int K = c->tree.depth;
+        const size_t Ka = m.n_medusa ? m.n_medusa : 1;  // heads the per-sequence buffers are laid out for
+        if (K > 0) {
+            cudaError_t e = cudaSuccess;
+            PROF(c, PC_HEADS, 1, e = launch_heads_resblock_batch(m.dtype, c->h_last_all, m.d, c->w.medusa_w1, c->head_x_all,
+                                                                 (long long)(Ka * m.d), K, m.d, B, c->stream));
+            if (e == cudaSuccess)
+                PROF(c, PC_HEADS, 1, e = launch_heads_vocab_batch(m.dtype, c->head_x_all, (long long)(Ka * m.d), c->w.medusa_w2,
+                                                                  c->head_logits_all, (long long)(Ka * m.vocab), K, m.d, m.vocab, B,
+                                                                  c->stream));
+            if (e != cudaSuccess) rc = fail(c, MEDUSA_ERR_CUDA, "batched heads launch failed: %s", cudaGetErrorString(e));
+        }
+        for (int b = 0; b < B && rc == MEDUSA_OK; ++b) {
+            point_at(c, b);
+            if (K > 0)
+                PROF(c, PC_TOPK, c->tree.topk <= 8 ? 2 : 1,
+                     launch_topk(c->head_logits, K, m.vocab, c->tree.topk, c->topk_idx, nullptr, c->topk_scratch, c->stream));
+            PROF(c, PC_TOPK, 1, launch_expand(c->d_state + ST_ROOT, c->topk_idx, c->d_tree_idx, c->tree_tok + (size_t)b * TREE_ROWS,
+                                              c->tree.T, c->stream));
+            if (cudaGetLastError() != cudaSuccess) rc = fail(c, MEDUSA_ERR_CUDA, "top-k / expansion launch failed");
+        }
     }
     // (2) one backbone pass over all sequences' tiles
     if (rc == MEDUSA_OK) rc = tree_pass(c, c->tree_tok, T, c->d_mask, c->d_pos, 0, c->tree.mask_words, B);

@@ -77,6 +77,11 @@ struct Args {
     const int32_t *cache_len;
     const uint64_t *mask;            // [T][mask_words]: bit j of row i -- tree node j visible to query i
     int mask_words;                  // 64 tree nodes per word (1 unless the kernel is instantiated with LARGE)
+    // LARGE instantiation only.  batch != 0: blockIdx.z is a SEQUENCE (one tile of 64 query rows each, all with the same
+    // tree of T nodes): its keys are its own cache (cache_seq_stride elements after the previous sequence's), its own
+    // cache length (len_stride ints after the previous one's) and its own tile of tree keys.
+    int batch, len_stride;
+    long long cache_seq_stride;
     bf16 *out, *out_lo;              // [T][H][D]; out_lo nullable
     float *lse;                      // nullable [T][H]
     float *ws_o;                     // [q tiles][H][max_splits][64][128] unnormalised partial outputs
@@ -343,14 +348,20 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     uint8_t *smem = smem_all + (QLO ? 2 : 1) * TILE_BYTES;  // K/V ring; the Q tile(s) sit in front of it
     __shared__ int s_ticket;
     const int h = blockIdx.x, sp = blockIdx.y;
+    const bool batch = LARGE && a.batch != 0;
     const int q0 = LARGE ? (int)blockIdx.z * BQ : 0;            // first query row of this CTA's tile
-    const int Tq = LARGE ? min(BQ, a.T - q0) : a.T;             // its query rows
-    const int tree_tiles = LARGE ? (int)blockIdx.z + 1 : 1;     // key tiles of the tree this query tile can see
+    const int Tq = LARGE && !batch ? min(BQ, a.T - q0) : a.T;   // its query rows
+    const int tree_tiles = LARGE && !batch ? (int)blockIdx.z + 1 : 1;  // key tiles of the tree this query tile can see
+    const int tree_tile0 = batch ? (int)blockIdx.z : 0;         // the first of them (a sequence's own tile in a batch)
+    const int mrow0 = batch ? 0 : q0;                           // mask row of the tile's first query
     const size_t slot = LARGE ? (size_t)blockIdx.z * a.H + h : (size_t)h;  // (query tile, head)
+    const bf16 *const kc_base = a.k_cache + (batch ? (size_t)blockIdx.z * a.cache_seq_stride : 0);
+    const bf16 *const vc_base = a.v_cache + (batch ? (size_t)blockIdx.z * a.cache_seq_stride : 0);
+    const int32_t *const len_ptr = a.cache_len + (batch ? (size_t)blockIdx.z * a.len_stride : 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
     const int wq = warp & 3, kh = warp >> 2;  // query-row group, key half
     // a length outside [0, L_max] would index past the caches: clamp (the driver's own state never leaves that range)
-    const int L = min(max(*a.cache_len, 0), a.L_max);
+    const int L = min(max(*len_ptr, 0), a.L_max);
     const int nt = (L + BKEY - 1) / BKEY;
     if (!LARGE && nt <= a.rows_max_tiles && gridDim.y >= 2) {
         if (sp < 2)
@@ -387,11 +398,11 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
         const int ct = tile0 + i;
         if (ct < tile1) {
             const size_t base = ((size_t)hk * a.L_max + (size_t)ct * BKEY) * D;
-            load_tile(stage, a.k_cache + base, a.v_cache + base, D, min(BKEY, L - ct * BKEY));
+            load_tile(stage, kc_base + base, vc_base + base, D, min(BKEY, L - ct * BKEY));
         } else {
-            const int w = LARGE ? ct - tile1 : 0;  // key tile of the tree
+            const int w = LARGE ? tree_tile0 + ct - tile1 : 0;  // key tile of the tree (row tile of k_new / v_new)
             const size_t tb = ((size_t)w * BKEY * a.Hkv + hk) * D;
-            load_tile(stage, a.k_new + tb, a.v_new + tb, HkvD, min(BKEY, a.T - w * BKEY));
+            load_tile(stage, a.k_new + tb, a.v_new + tb, HkvD, batch ? a.T : min(BKEY, a.T - w * BKEY));
         }
     };
     // ---- Q and the first K/V tiles are requested together; Q is copy group 0
@@ -428,8 +439,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
     const int row0 = wq * 16 + g, row1 = row0 + 8;  // rows inside the query tile
     // mask words of this thread's two rows for the tree's first key tile; with LARGE the words of the following key tiles
     // are fetched one tile ahead inside the loop
-    uint64_t mask0 = row0 < Tq ? a.mask[(size_t)(q0 + row0) * (LARGE ? a.mask_words : 1)] : 0ull;
-    uint64_t mask1 = row1 < Tq ? a.mask[(size_t)(q0 + row1) * (LARGE ? a.mask_words : 1)] : 0ull;
+    uint64_t mask0 = row0 < Tq ? a.mask[(size_t)(mrow0 + row0) * (LARGE ? a.mask_words : 1)] : 0ull;
+    uint64_t mask1 = row1 < Tq ? a.mask[(size_t)(mrow0 + row1) * (LARGE ? a.mask_words : 1)] : 0ull;
     uint64_t next_mask0 = 0ull, next_mask1 = 0ull;
     const float sc = rsqrtf((float)D) * LOG2E;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
@@ -479,8 +490,8 @@ __global__ void __launch_bounds__(THREADS, 1) tree_attention_flash_kernel(Args a
             const int w = ct - tile1;
             if (w > 0) { mask0 = next_mask0; mask1 = next_mask1; }
             if (w + 1 < tree_tiles) {
-                if (row0 < Tq) next_mask0 = a.mask[(size_t)(q0 + row0) * a.mask_words + w + 1];
-                if (row1 < Tq) next_mask1 = a.mask[(size_t)(q0 + row1) * a.mask_words + w + 1];
+                if (row0 < Tq) next_mask0 = a.mask[(size_t)(mrow0 + row0) * a.mask_words + w + 1];
+                if (row1 < Tq) next_mask1 = a.mask[(size_t)(mrow0 + row1) * a.mask_words + w + 1];
             }
         }
 #pragma unroll
@@ -772,7 +783,8 @@ static cudaError_t flash_set_limits()
 cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                        int L_hint, cudaStream_t s, const void *q_lo, int mask_words)
+                                        int L_hint, cudaStream_t s, const void *q_lo, int mask_words, int n_seq,
+                                        long long cache_seq_stride, int len_stride)
 {
     {
         cudaError_t e = flash_set_limits();
@@ -794,8 +806,12 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
         }
     }
     Args a;
-    const int q_tiles = (T + BQ - 1) / BQ;
+    // n_seq > 1: a batch of sequences, one tile of 64 query rows each (T <= 64 is then the tree size of every sequence)
+    const int q_tiles = n_seq > 1 ? n_seq : (T + BQ - 1) / BQ;
     const bool large = q_tiles > 1, qlo = q_lo != nullptr;
+    a.batch = n_seq > 1 ? 1 : 0;
+    a.cache_seq_stride = cache_seq_stride;
+    a.len_stride = len_stride;
     const size_t slots = (size_t)H * q_tiles;
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
     a.q_lo = (const bf16 *)q_lo;
@@ -884,6 +900,7 @@ extern "C" int32_t medusa_tree_attention_static(const void *q, const void *k_new
     Args a;
     a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
     a.q_lo = nullptr;
+    a.batch = 0; a.len_stride = 0; a.cache_seq_stride = 0;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
     a.cache_len = cache_len; a.mask = mask; a.mask_words = 1; a.out = (bf16 *)out; a.out_lo = nullptr; a.lse = lse;
     a.ws_o = base;

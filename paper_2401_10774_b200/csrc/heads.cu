@@ -117,6 +117,131 @@ static void launch_gemv(const WT *W, const XT *x, int x_head_stride, float *out,
     launch_pdl(gemv_kernel<WT, XT, EPI>, dim3(blocks, K), dim3(GV_WARPS * 32), smem, s, W, x, x_head_stride, out, rows, d);
 }
 
+// ---------------------------------------------------------------------------------------- batched GEMV (batch > 1)
+// The same products for up to GVB_MAX sequences at once: every weight row is loaded once and multiplied with all the
+// sequences' input vectors (held side by side in shared memory), so a batched step streams the head weights once.
+// Sums per (row, sequence) are formed in the same order as in the single-sequence kernel.
+constexpr int GVB_MAX = 4;
+
+template <typename WT, int EPI, int NR>
+__device__ __forceinline__ void gemv_rows_batch(const WT *__restrict__ Wh, const float *__restrict__ xs, float *__restrict__ out_h,
+                                                long long out_batch_stride, int row, int d, int nb, int lane)
+{
+    constexpr int VN = Vec16<WT>::N;
+    float acc[NR][GVB_MAX];
+#pragma unroll
+    for (int r = 0; r < NR; ++r)
+#pragma unroll
+        for (int b = 0; b < GVB_MAX; ++b)
+            acc[r][b] = 0.f;
+    const WT *w0 = Wh + (size_t)row * d;
+    const int chunks = d / VN;
+    for (int c = lane; c < chunks; c += 32) {
+        float wv[NR][VN];
+#pragma unroll
+        for (int r = 0; r < NR; ++r)
+            Vec16<WT>::load(w0 + (size_t)r * d + (size_t)c * VN, wv[r]);
+#pragma unroll
+        for (int b = 0; b < GVB_MAX; ++b) {
+            if (b < nb) {
+                float xv[VN];
+#pragma unroll
+                for (int e = 0; e < VN; e += 4) {
+                    float4 t = *reinterpret_cast<const float4 *>(xs + (size_t)b * d + c * VN + e);
+                    xv[e] = t.x; xv[e + 1] = t.y; xv[e + 2] = t.z; xv[e + 3] = t.w;
+                }
+#pragma unroll
+                for (int r = 0; r < NR; ++r)
+#pragma unroll
+                    for (int e = 0; e < VN; ++e)
+                        acc[r][b] = fmaf(wv[r][e], xv[e], acc[r][b]);
+            }
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < GVB_MAX; ++b) {
+        if (b < nb) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r)
+                acc[r][b] = warp_sum(acc[r][b]);
+            if (lane < NR) {
+                float y = acc[0][b];
+#pragma unroll
+                for (int r = 1; r < NR; ++r)
+                    if (lane == r)
+                        y = acc[r][b];
+                out_h[(size_t)b * out_batch_stride + row + lane] = EPI == GV_LOGITS ? y : xs[(size_t)b * d + row + lane] + silu_f(y);
+            }
+        }
+    }
+}
+
+// x: float, sequence b's vector of head k at x + b * x_batch_stride + k * x_head_stride; out[b][k][rows] with
+// out_batch_stride floats between sequences
+template <typename WT, int EPI>
+__global__ void __launch_bounds__(GV_WARPS * 32)
+gemv_batch_kernel(const WT *__restrict__ W, const float *__restrict__ x, int x_head_stride, long long x_batch_stride,
+                  float *__restrict__ out, long long out_batch_stride, int rows, int d, int nb)
+{
+    pdl_enter();
+    extern __shared__ float xs[];  // [nb][d]
+    const int head = blockIdx.y;
+    for (int b = 0; b < nb; ++b) {
+        const float *xh = x + (size_t)b * x_batch_stride + (size_t)head * x_head_stride;
+        for (int i = threadIdx.x; i < d; i += blockDim.x)
+            xs[(size_t)b * d + i] = xh[i];
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long w = (long long)blockIdx.x * GV_WARPS + warp, n_warps = (long long)gridDim.x * GV_WARPS;
+    int row = (int)(w * rows / n_warps);
+    const int row_end = (int)((w + 1) * rows / n_warps);
+    const WT *Wh = W + (size_t)head * rows * d;
+    float *out_h = out + (size_t)head * rows;
+    for (; row + 2 <= row_end; row += 2)
+        gemv_rows_batch<WT, EPI, 2>(Wh, xs, out_h, out_batch_stride, row, d, nb, lane);
+    if (row < row_end)
+        gemv_rows_batch<WT, EPI, 1>(Wh, xs, out_h, out_batch_stride, row, d, nb, lane);
+}
+
+template <typename WT, int EPI>
+static cudaError_t launch_gemv_batch(const WT *W, const float *x, int x_head_stride, long long x_batch_stride, float *out,
+                                     long long out_batch_stride, int rows, int d, int K, int nb, cudaStream_t s)
+{
+    const size_t smem = (size_t)nb * d * sizeof(float);
+    static bool attr[64] = {};
+    if (first_use_on_current_device(attr)) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_batch_kernel<WT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess)
+            return e;
+    }
+    const int blocks = gemv_blocks_per_head(gemv_batch_kernel<WT, EPI>, smem, rows, K);
+    return launch_pdl(gemv_batch_kernel<WT, EPI>, dim3(blocks, K), dim3(GV_WARPS * 32), smem, s, W, x, x_head_stride, x_batch_stride,
+                      out, out_batch_stride, rows, d, nb);
+}
+
+// h_all: float [nb][d] (h_stride floats apart); x_all: float out, sequence b's [K][d] block x_stride floats after b-1's
+cudaError_t launch_heads_resblock_batch(int dtype, const float *h_all, long long h_stride, const void *W1, float *x_all,
+                                        long long x_stride, int K, int d, int nb, cudaStream_t s)
+{
+    if (nb < 1 || nb > GVB_MAX)
+        return cudaErrorInvalidValue;
+    if (dtype == MEDUSA_BF16)
+        return launch_gemv_batch<bf16, GV_RESBLOCK>((const bf16 *)W1, h_all, 0, h_stride, x_all, x_stride, d, d, K, nb, s);
+    return launch_gemv_batch<float, GV_RESBLOCK>((const float *)W1, h_all, 0, h_stride, x_all, x_stride, d, d, K, nb, s);
+}
+
+// x_all as above; logits_all: float out, sequence b's [K][V] block z_stride floats after b-1's
+cudaError_t launch_heads_vocab_batch(int dtype, const float *x_all, long long x_stride, const void *W2, float *logits_all,
+                                     long long z_stride, int K, int d, int V, int nb, cudaStream_t s)
+{
+    if (nb < 1 || nb > GVB_MAX)
+        return cudaErrorInvalidValue;
+    if (dtype == MEDUSA_BF16)
+        return launch_gemv_batch<bf16, GV_LOGITS>((const bf16 *)W2, x_all, d, x_stride, logits_all, z_stride, V, d, K, nb, s);
+    return launch_gemv_batch<float, GV_LOGITS>((const float *)W2, x_all, d, x_stride, logits_all, z_stride, V, d, K, nb, s);
+}
+
 void launch_heads_resblock(int dtype, const void *h, int h_is_f32, const void *W1, float *x, int K, int d, cudaStream_t s)
 {
     if (dtype == MEDUSA_BF16 && !h_is_f32)

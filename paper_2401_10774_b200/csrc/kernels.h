@@ -57,11 +57,15 @@ size_t tree_attention_flash_workspace_bytes(int H, int q_tiles = 1);  // q_tiles
 // same contract as the kernel above; L_hint: host-side upper bound of *cache_len (the tcgen05 kernel sizes its grid
 // with it; the mma.sync kernel picks its key ranges from *cache_len on the device);
 // workspace: tree_attention_flash_workspace_bytes(H) bytes, zero-initialised once
-// q_lo (nullable): second plane of q; with it the scores are q.k + q_lo.k
+// q_lo (nullable): second plane of q; with it the scores are q.k + q_lo.k.
+// n_seq > 1: a batch -- q, k_new, v_new, out hold n_seq tiles of 64 rows (sequence b at rows 64 b..), every sequence with
+// the same tree of T <= 64 nodes; sequence b's caches start cache_seq_stride elements after sequence b-1's and its cache
+// length len_stride ints after sequence b-1's; the workspace must have been sized for n_seq query tiles.
 cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                         const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                         void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                        int L_hint, cudaStream_t s, const void *q_lo = nullptr, int mask_words = 1);
+                                        int L_hint, cudaStream_t s, const void *q_lo = nullptr, int mask_words = 1,
+                                        int n_seq = 1, long long cache_seq_stride = 0, int len_stride = 0);
 // The same operation and workspace on the tcgen05 tensor cores (attention_tc.cu): scores and P V accumulate in
 // TMEM, softmax threads own one query row each.  status: device status word (MEDUSA_ERR_TIMEOUT on an expired wait).
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,
@@ -72,6 +76,13 @@ cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const voi
 // ---- heads.cu ----
 // x_k = h + SiLU(W1_k h) -> float [K][d];  h: float if h_is_f32 else the model dtype
 void launch_heads_resblock(int dtype, const void *h, int h_is_f32, const void *W1, float *x, int K, int d, cudaStream_t s);
+// the same two products for nb <= 4 sequences at once (batch > 1): every weight row is read once for all of them.
+// h_all: float [nb][d] (h_stride floats apart); x_all: sequence b's float [K][d] block x_stride floats after b-1's;
+// logits_all: sequence b's float [K][V] block z_stride floats after b-1's
+cudaError_t launch_heads_resblock_batch(int dtype, const float *h_all, long long h_stride, const void *W1, float *x_all,
+                                        long long x_stride, int K, int d, int nb, cudaStream_t s);
+cudaError_t launch_heads_vocab_batch(int dtype, const float *x_all, long long x_stride, const void *W2, float *logits_all,
+                                     long long z_stride, int K, int d, int V, int nb, cudaStream_t s);
 // z_k = W2_k x_k  -> logits float [K][V]
 void launch_heads_vocab(int dtype, const float *x, const void *W2, float *logits, int K, int d, int V, cudaStream_t s);
 // per head: indices of the topk largest (value desc, index asc)
