@@ -130,10 +130,14 @@ enum {
                                       * buffers (parity checks layer by layer); -1 (default) off */
     MEDUSA_OPT_SPIN_LIMIT = 4,       /* polls after which a bounded device-side wait gives up with MEDUSA_ERR_TIMEOUT;
                                       * 0 = the kernels' default (about 4 million) */
-    MEDUSA_OPT_WITHHOLD_LOAD = 5     /* failure-path test hook, one shot: 1 = in the next tensor-core GEMM launch, 2 = in the
+    MEDUSA_OPT_WITHHOLD_LOAD = 5,    /* failure-path test hook, one shot: 1 = in the next tensor-core GEMM launch, 2 = in the
                                       * next tcgen05 attention launch, one CTA's producer issues no load at all, so that its
                                       * consumers' bounded waits expire with nothing in flight; the launch returns, its output
                                       * is unusable and the device status becomes MEDUSA_ERR_TIMEOUT */
+    MEDUSA_OPT_ACTIVATION_PLANES = 6  /* bf16 model: planes of every activation the projections read.  2 (default): a value
+                                       * y is held as hi = bf16(y) and lo = bf16(y - hi) and a projection is W hi + W lo
+                                       * (accurate to ~2^-17); 1: hi only -- half the tensor-core work and up to 256 token
+                                       * rows per weight stream (large trees, batches), at bf16 accuracy of the inputs */
 };
 
 /* ---- lifetime ------------------------------------------------------------------------------------ */

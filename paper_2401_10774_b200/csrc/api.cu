@@ -81,7 +81,12 @@ struct medusa_ctx {
     bool use_tc = false;
     TensorMap map_xn, map_att, map_act, map_hidden, map_lm;
     std::vector<TensorMap> wmaps;  // per layer: wq, wk, wv, wo, w_gate, w_up, w_down
-    void *lo(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 ? (char *)hi + (size_t)rows * width * 2 : nullptr; }
+    // activation planes the projections read (MEDUSA_OPT_ACTIVATION_PLANES): 2 = hi + lo (default), 1 = hi only
+    int act_planes = 2;
+    // the lo plane of a split activation (null in the f32 model and when the projections read one plane only)
+    void *lo(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 && act_planes == 2 ? (char *)hi + (size_t)rows * width * 2 : nullptr; }
+    // the second plane of q, which the attention kernel reads whatever the projections do
+    void *q_lo_plane(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 ? (char *)hi + (size_t)rows * width * 2 : nullptr; }
     float *logits = nullptr, *head_logits = nullptr;
     float2 *rope_cs = nullptr;
     void *tree_k = nullptr, *tree_v = nullptr, *k_cache = nullptr, *v_cache = nullptr;
@@ -275,8 +280,8 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
         const TensorMap *maps[3] = {mapW, mapW + (n_seg > 1 ? 1 : 0), mapW + (n_seg > 2 ? 2 : 0)};
         // up to 64 rows: one launch of one token tile; more: launches of two token tiles (128 rows) each, so that the
         // weights are streamed once per 128 rows
-        const int RT = gemm_tc_row_tiles(T), rows_per_launch = RT * TREE_ROWS;
-        *pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, (long long)plane_stride, seg0_cols, RT);
+        const int RT = gemm_tc_row_tiles(T, c->act_planes), rows_per_launch = RT * TREE_ROWS;
+        *pd = gemm_tc_plan(n_seg, seg_cols, K, whole_tiles, (long long)plane_stride, seg0_cols, RT, c->act_planes);
         if (!whole_tiles && (size_t)pd->n_max * plane_stride > c->part_elems)
             return fail(c, MEDUSA_ERR_SHAPE, "projection needs %d partial planes, more than the workspace holds", pd->n_max);
         // every launch of the projection uses the same plan, so the consumer finds the same pieces in every row
@@ -286,7 +291,7 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
             if (wh) c->withhold = 0;
             const int Tt = T - r0 < rows_per_launch ? T - r0 : rows_per_launch, row0t = row0 > r0 ? row0 - r0 : 0;
             PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, n_seg, seg_cols, K, *pd, P + (size_t)r0 * ldy, ldy, Tt, row0t,
-                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0, RT));
+                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0, RT, c->act_planes));
             if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "tensor-core GEMM launch failed: %s", cudaGetErrorString(e));
         }
         return MEDUSA_OK;
@@ -353,7 +358,7 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
         if (Hkv == H || !c->use_tc || (HD % 128 == 0 && HkvD % 128 == 0)) {
             // one launch for [q | k | v]; with grouped-query attention the k and v matrices are narrower than q
             TRY(project(c, c->xn, &c->map_xn, wqkv, wm, 3, HkvD, d, c->part, (size_t)c->rows * qkv_ld, qkv_ld, T, 0, false, &pd, HD));
-            PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd, 0, c->rope_cs, c->q, c->lo(c->q, HD), tk, tv, T, H, Hkv, D, s));
+            PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd, 0, c->rope_cs, c->q, c->q_lo_plane(c->q, HD), tk, tv, T, H, Hkv, D, s));
         } else {
             // widths that are not multiples of the 128-row tile: q alone (any width), then k and v on the CUDA-core
             // kernel, into disjoint columns of the same rows
@@ -361,7 +366,7 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
             TRY(project(c, c->xn, &c->map_xn, wqkv, wm, 1, HD, d, c->part, (size_t)c->rows * qkv_ld, qkv_ld, T, 0, false, &pd));
             TRY(project(c, c->xn, &c->map_xn, wqkv + 1, wm ? wm + 1 : nullptr, 2, HkvD, d, c->part + HD, (size_t)c->rows * qkv_ld,
                         qkv_ld, T, 0, false, &pd_kv));
-            PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd_kv, HD, c->rope_cs, c->q, c->lo(c->q, HD), tk, tv, T, H, Hkv, D, s));
+            PROF(c, PC_ELEMWISE, 1, launch_rope_split(dt, c->part, pd, pd_kv, HD, c->rope_cs, c->q, c->q_lo_plane(c->q, HD), tk, tv, T, H, Hkv, D, s));
         }
         MEDUSA_LAUNCH_CHECK(c);
         if (n_seq > 1 && c->flash_ws && c->attn_mode != 2) {
@@ -370,7 +375,7 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
             const size_t lay = (size_t)l * Hkv * m.L_max * D * c->esz;
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_flash(c->q, tk, tv, c->k_cache_all + lay, c->v_cache_all + lay,
                                                                      c->state_all + ST_CACHE_LEN, mask, c->att, c->lo(c->att, HD), nullptr,
-                                                                     c->flash_ws, T_seq, H, Hkv, m.L_max, m.L_max, s, c->lo(c->q, HD),
+                                                                     c->flash_ws, T_seq, H, Hkv, m.L_max, m.L_max, s, c->q_lo_plane(c->q, HD),
                                                                      mask_words, n_seq, (long long)(c->cache_seq_bytes / c->esz), ST_WORDS));
             if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "batched flash attention launch failed: %s", cudaGetErrorString(e));
         } else if (n_seq > 1) {
@@ -379,7 +384,7 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
             for (int b = 0; b < n_seq; ++b) {
                 const size_t ro = (size_t)b * TREE_ROWS;  // first row of the sequence
                 const size_t lay = (size_t)l * Hkv * m.L_max * D * c->esz;
-                const char *q_lo = (const char *)c->lo(c->q, HD);
+                const char *q_lo = (const char *)c->q_lo_plane(c->q, HD);
                 char *att_lo = (char *)c->lo(c->att, HD);
                 TRY(attention(c, (const char *)c->q + ro * HD * c->esz, tk + ro * HkvD * c->esz, tv + ro * HkvD * c->esz,
                               c->k_cache_all + (size_t)b * c->cache_seq_bytes + lay, c->v_cache_all + (size_t)b * c->cache_seq_bytes + lay,
@@ -389,7 +394,7 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
             }
         } else {
             TRY(attention(c, c->q, tk, tv, kc, vc, cache_len, mask, c->att, c->lo(c->att, HD), nullptr, T, c->L_upper, true,
-                          mask_words, c->lo(c->q, HD)));
+                          mask_words, c->q_lo_plane(c->q, HD)));
         }
         if (l == c->tap_layer)
             MEDUSA_CUDA(c, cudaMemcpyAsync(c->tap_att, c->att, (dt == MEDUSA_BF16 ? 2 : 1) * (size_t)c->rows * HD * c->esz,
@@ -693,6 +698,13 @@ extern "C" int32_t medusa_set_option(medusa_ctx *c, int32_t option, int64_t valu
         MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
         drop_step_graphs(c);  // captured launches carry the old limit
         c->spin_limit = (uint32_t)value;
+        return MEDUSA_OK;
+    case MEDUSA_OPT_ACTIVATION_PLANES:
+        if (value != 1 && value != 2) return fail(c, MEDUSA_ERR_INVALID_ARG, "activation planes: 1 or 2");
+        MEDUSA_CUDA(c, cudaSetDevice(c->device));
+        MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
+        drop_step_graphs(c);
+        c->act_planes = (int)value;
         return MEDUSA_OK;
     case MEDUSA_OPT_WITHHOLD_LOAD:
         if (value < 0 || value > 2) return fail(c, MEDUSA_ERR_INVALID_ARG, "withhold: 0 (off), 1 (next tensor-core GEMM) or 2 (next tcgen05 attention)");

@@ -34,15 +34,16 @@ namespace {
 
 constexpr int BM = 128;                 // weight rows per tile (UMMA M)
 constexpr int BN = 64;                  // tokens
-constexpr int UMMA_N = 2 * BN;          // MMA N: the hi plane's 64 token rows followed by the lo plane's
+// MMA N per token tile: PL * BN -- the hi plane's 64 token rows, followed by the lo plane's when the activations come as
+// two planes (PL = 2)
 constexpr int BK = 64;                  // k elements per stage: one 128-byte swizzle row of bf16
 constexpr int UMMA_K = 16;
 constexpr int MAX_STAGES = 8;         // ring depth is a launch parameter (a.stages)
 constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;    // 8 KiB per plane
-// a stage: one weight tile and, for each of the launch's RT token tiles, the two activation planes
-constexpr int stage_bytes(int rt) { return A_BYTES + rt * 2 * B_BYTES; }
-constexpr int smem_bytes(int stages, int rt) { return stages * stage_bytes(rt) + 1024 /* alignment slack */ + 256 /* barriers */; }
+// a stage: one weight tile and, for each of the launch's RT token tiles, the PL activation planes
+constexpr int stage_bytes(int rt, int pl) { return A_BYTES + rt * pl * B_BYTES; }
+constexpr int smem_bytes(int stages, int rt, int pl) { return stages * stage_bytes(rt, pl) + 1024 /* alignment slack */ + 256 /* barriers */; }
 constexpr int THREADS = 192;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -98,12 +99,13 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr)
     return d;
 }
 
-// instruction descriptor: D fp32, A and B bf16, both K-major, N = 128, M = 128
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(UMMA_N >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// instruction descriptor: D fp32, A and B bf16, both K-major, N = n, M = 128
+constexpr uint32_t idesc(int n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24); }
 
 // The MMA warp runs its loop convergently (descriptor arithmetic stays warp-uniform); the tcgen05 instructions
 // are predicated on `leader` (lane 0) instead of sitting in a divergent branch.
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate, uint32_t leader)
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t IDESC, uint32_t accumulate,
+                                     uint32_t leader)
 {
     asm volatile("{\n\t.reg .pred p, q;\n\t"
                  "setp.ne.b32 p, %4, 0;\n\t"
@@ -193,18 +195,21 @@ struct SegmentIter {
     }
 };
 
-// RT = token tiles (64 rows each) per launch.  RT = 1: two CTAs per SM, two 128-column accumulators each.  RT = 2 (trees
-// of more than 64 nodes): the weight tile of a stage feeds two MMAs, one per token tile, into two accumulators; a CTA then
-// holds all 512 tensor-memory columns (2 buffers x 2 tiles x 128), so one CTA per SM with a deeper ring.
-template <int RT>
-__global__ void __launch_bounds__(THREADS, RT == 1 ? 2 : 1)
+// RT = token tiles (64 rows each) per launch, PL = activation planes (2: hi + lo, the default; 1: hi only).  The weight
+// tile of a stage feeds RT MMAs of N = 64 PL, one per token tile, into RT accumulators of 64 PL columns; the accumulators
+// are double-buffered, so a CTA holds 2 RT 64 PL tensor-memory columns: up to 256 leaves room for two CTAs per SM,
+// 512 (RT PL = 4) means one CTA per SM with a deeper ring.
+template <int RT, int PL>
+__global__ void __launch_bounds__(THREADS, RT * PL <= 2 ? 2 : 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW0,
                const __grid_constant__ CUtensorMap mapW1, const __grid_constant__ CUtensorMap mapW2, GemmTcArgs a)
 {
-    constexpr int STAGE_BYTES = stage_bytes(RT);
+    constexpr int STAGE_BYTES = stage_bytes(RT, PL);
+    constexpr int UMMA_N = PL * BN;              // MMA N of one token tile
+    constexpr uint32_t IDESC = idesc(UMMA_N);
     constexpr uint32_t ACC_COLS = RT * UMMA_N;   // columns of one accumulator set (all token tiles of a segment)
     const int rt_n = min(RT, (a.T + BN - 1) / BN);  // token tiles that hold rows in this launch
-    const uint32_t stage_tx = (uint32_t)(A_BYTES + rt_n * 2 * B_BYTES);
+    const uint32_t stage_tx = (uint32_t)(A_BYTES + rt_n * PL * B_BYTES);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the next kernel may start its prologue
     extern __shared__ uint8_t smem_raw[];
     // tiles must sit on 1024-byte boundaries for the 128-byte swizzle pattern
@@ -250,8 +255,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             // the activation planes of k block `k` for every token tile of the launch: hi rows, then lo rows
             auto load_x = [&](uint8_t *st, int k, uint64_t *bar) {
                 for (int rt = 0; rt < rt_n; ++rt) {
-                    tma_load_2d(st + A_BYTES + rt * 2 * B_BYTES, &mapX, k, a.x_row_hi + rt * BN, bar, pol_keep);
-                    tma_load_2d(st + A_BYTES + rt * 2 * B_BYTES + B_BYTES, &mapX, k, a.x_row_lo + rt * BN, bar, pol_keep);
+                    tma_load_2d(st + A_BYTES + rt * PL * B_BYTES, &mapX, k, a.x_row_hi + rt * BN, bar, pol_keep);
+                    if (PL == 2)
+                        tma_load_2d(st + A_BYTES + rt * PL * B_BYTES + B_BYTES, &mapX, k, a.x_row_lo + rt * BN, bar, pol_keep);
                 }
             };
             SegmentIter it(a, blockIdx.x);
@@ -334,11 +340,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
 #pragma unroll
                     for (int rt = 0; rt < RT; ++rt) {
                         if (rt < rt_n) {
-                            const uint64_t db = umma_desc(sa + A_BYTES + rt * 2 * B_BYTES);
+                            const uint64_t db = umma_desc(sa + A_BYTES + rt * PL * B_BYTES);
 #pragma unroll
                             for (int k = 0; k < BK / UMMA_K; ++k) {
                                 const uint64_t adv = (uint64_t)((k * UMMA_K * 2) >> 4);  // 32 bytes per step inside the swizzled row
-                                umma(tmem_d + (uint32_t)(rt * UMMA_N), da + adv, db + adv, (i | k) ? 1u : 0u, leader);
+                                umma(tmem_d + (uint32_t)(rt * UMMA_N), da + adv, db + adv, IDESC, (i | k) ? 1u : 0u, leader);
                             }
                         }
                     }
@@ -385,8 +391,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     uint32_t v[32], w[32];
                     const uint32_t col = (uint32_t)b * ACC_COLS + (uint32_t)(rt * UMMA_N + half * 32);
                     tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col, v);
-                    tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col + BN, w);
+                    if (PL == 2)
+                        tmem_ld32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + col + BN, w);
                     tmem_ld_wait();
+                    if (PL == 1) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            w[i] = 0u;  // +0.0f
+                    }
                     if (n_ok) {
                         float *o = out + (size_t)(tb + half * 32) * a.ldy;  // a warp writes 32 consecutive floats per token row
                         if (all_rows) {
@@ -484,12 +496,19 @@ int gemm_tc_stages()
     return v;
 }
 
-// Token tiles per launch: one for up to 64 rows, two for more (the weight stream then serves both tiles).
-int gemm_tc_row_tiles(int T) { return T > BN ? 2 : 1; }
-// ring depth of the two-tile form (one CTA per SM, 48 KiB per stage)
-static int gemm_tc_stages_rt2() { return 4; }
+// Token tiles per launch: one for up to 64 rows, two for more (the weight stream then serves both tiles); with a
+// single activation plane four tiles fit the tensor memory, so up to 256 rows share one weight stream.
+int gemm_tc_row_tiles(int T, int planes) { return T > 2 * BN && planes == 1 ? 4 : (T > BN ? 2 : 1); }
+// CTAs per SM and ring depth by (token tiles, planes): two CTAs per SM while 2 * RT * PL * 64 columns fit 256
+static int cfg_ctas_per_sm(int rt, int pl) { return rt * pl <= 2 ? gemm_tc_ctas_per_sm() : 1; }
+static int cfg_stages(int rt, int pl)
+{
+    if (rt == 1 && pl == 2) return gemm_tc_stages();  // 32 KiB stages, the tuned default
+    if (rt * pl <= 2) return rt == 1 ? 4 : 3;         // (1,1): 24 KiB x 4;  (2,1): 32 KiB x 3
+    return 4;                                         // (2,2) and (4,1): 48 KiB x 4, one CTA per SM
+}
 
-int gemm_tc_num_ctas(int row_tiles)
+int gemm_tc_num_ctas(int row_tiles, int planes)
 {
     static int sms = 0;
     if (!sms) {
@@ -498,17 +517,18 @@ int gemm_tc_num_ctas(int row_tiles)
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             sms = 148;
     }
-    return sms * (row_tiles > 1 ? 1 : gemm_tc_ctas_per_sm());
+    return sms * cfg_ctas_per_sm(row_tiles, planes);
 }
 
-PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols, int row_tiles)
+PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols, int row_tiles,
+                       int planes)
 {
     PlaneDesc pd{};
     if (seg0_cols <= 0) seg0_cols = seg_cols;
     const int tiles = (seg0_cols + BM - 1) / BM + (n_seg - 1) * ((seg_cols + BM - 1) / BM);
     const int KB = (K + BK - 1) / BK;
     const long long total = (long long)tiles * KB;
-    int G = gemm_tc_num_ctas(row_tiles);
+    int G = gemm_tc_num_ctas(row_tiles, planes);
     if (whole_tiles) {
         if (G > tiles) G = tiles;
         pd.n_max = 1; pd.KB = KB; pd.G = 0; pd.total = total; pd.stride = plane_stride; pd.ctas = G;
@@ -524,19 +544,30 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
     return pd;
 }
 
+typedef void (*GemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, GemmTcArgs);
+static GemmKernel gemm_kernel(int rt, int pl)
+{
+    if (pl == 2) return rt == 1 ? gemm_tc_kernel<1, 2> : gemm_tc_kernel<2, 2>;
+    return rt == 1 ? gemm_tc_kernel<1, 1> : (rt == 2 ? gemm_tc_kernel<2, 1> : gemm_tc_kernel<4, 1>);
+}
+
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
-                           int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo, int row_tiles)
+                           int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo, int row_tiles,
+                           int planes)
 {
     if (seg0_cols <= 0) seg0_cols = seg_cols;
-    const int stages = row_tiles > 1 ? gemm_tc_stages_rt2() : gemm_tc_stages();
+    const int rt = row_tiles >= 4 && planes == 1 ? 4 : (row_tiles >= 2 ? 2 : 1), pl = planes == 1 ? 1 : 2;
+    const int stages = cfg_stages(rt, pl);
     static bool attr_set[64] = {};
     if (first_use_on_current_device(attr_set)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(gemm_tc_stages(), 1));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(gemm_tc_stages_rt2(), 2));
-        if (e != cudaSuccess)
-            return e;
+        const int cfgs[5][2] = {{1, 2}, {2, 2}, {1, 1}, {2, 1}, {4, 1}};
+        for (auto &cf : cfgs) {
+            cudaError_t e = cudaFuncSetAttribute(gemm_kernel(cf[0], cf[1]), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 smem_bytes(cfg_stages(cf[0], cf[1]), cf[0], cf[1]));
+            if (e != cudaSuccess)
+                return e;
+        }
     }
     GemmTcArgs a;
     a.P = P;
@@ -564,16 +595,14 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(pd.ctas);
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = smem_bytes(a.stages, row_tiles > 1 ? 2 : 1);
+    cfg.dynamicSmemBytes = smem_bytes(stages, rt, pl);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = tuning_env("MEDUSA_NO_PDL") ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (row_tiles > 1)
-        return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1>, *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
+    return cudaLaunchKernelEx(&cfg, gemm_kernel(rt, pl), *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
 }
 
 }  // namespace medusa

@@ -60,22 +60,24 @@ struct GemmTcArgs {
 bool make_weight_map(TensorMap *out, const void *W, int N, int K);
 // X_planes: split activation, [2][rows][K] bf16 (hi plane, then lo plane; rows a multiple of 64)
 bool make_act_map(TensorMap *out, const void *X_planes, int K, int rows = 64);
-int gemm_tc_num_ctas(int row_tiles = 1);
-// token tiles (64 rows each) one launch covers for a pass over T rows: 1 up to 64 rows, 2 beyond
-int gemm_tc_row_tiles(int T);
+int gemm_tc_num_ctas(int row_tiles = 1, int planes = 2);
+// token tiles (64 rows each) one launch covers for a pass over T rows: 1 up to 64 rows, 2 beyond; 4 beyond 128 rows when
+// the activations come as a single plane (the accumulators of four tiles then fit the tensor memory)
+int gemm_tc_row_tiles(int T, int planes = 2);
 int gemm_tc_stages();
 int gemm_tc_ctas_per_sm();
 // plan of a launch over n_seg weight matrices of seg_cols rows (seg_cols % 128 == 0 unless n_seg == 1); the first
 // matrix has seg0_cols rows if that is given (> 0, a multiple of 128)
 PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long long plane_stride, int seg0_cols = 0,
-                       int row_tiles = 1);
+                       int row_tiles = 1, int planes = 2);
 // P[piece][t][first column of segment seg + n] = partial sums over k of (X_hi + X_lo)[t][k] * W_seg[n][k], t in [row0, T);
 // the launch's token rows t = 0.. are rows x_row_hi + t and x_row_lo + t of the activation tensor: 64 rows per launch
-// with row_tiles = 1, 128 with row_tiles = 2 (pd must come from gemm_tc_plan with the same row_tiles); a tree of more
+// with row_tiles = 1, 128 with row_tiles = 2, 256 with row_tiles = 4 (single plane only; pd must come from
+// gemm_tc_plan with the same row_tiles and planes); planes = 1: only the hi plane is read (P = X_hi * W); a tree of more
 // rows than one launch covers is projected launch by launch with P advanced accordingly
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
                            int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0, int x_row_hi = 0, int x_row_lo = 64,
-                           int row_tiles = 1);
+                           int row_tiles = 1, int planes = 2);
 
 }  // namespace medusa

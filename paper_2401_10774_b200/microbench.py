@@ -35,6 +35,7 @@ def main():
     ap.add_argument("--typical", action="store_true", help="typical acceptance (0.7 / 0.09 / 0.3) instead of greedy")
     ap.add_argument("--attention", type=int, default=0, metavar="L", help="time tree_attention alone at cache length L")
     ap.add_argument("--caches", type=int, default=32)
+    ap.add_argument("--planes", type=int, default=2, choices=(1, 2))
     ap.add_argument("--device-weights", action="store_true",
                     help="draw the weights on the device (N(0, 0.02^2), not the seeded host recipe): seconds instead of a "
                          "minute of set-up, for timing runs whose numbers do not depend on the values")
@@ -70,6 +71,8 @@ def main():
         dw["layers"] = [{k: dev(v) for k, v in lw.items()} for lw in w["layers"]]
     ctx = B.Context(cfg, B.BF16, args.L_max)
     ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
+    if args.planes != 2:
+        ctx.set_option(B.OPT_ACTIVATION_PLANES, args.planes)
     ctx.load_weights(dw)
     # a cache of the requested length without paying for a long prefill: prefill 64 tokens, then tell the
     # library the rest is there (the K/V values beyond are zeros, which is fine for timing)

@@ -205,3 +205,47 @@ def test_large_tree_bf16_decode_stagewise(oracle, mode):
         multi += n > 1
     assert multi > 0
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- projections on a single activation plane
+
+@pytest.mark.parametrize("tree_name,n_prompt", [("sparse64_d4", 70), ("sparse128_d4", 70), ("sparse256_d4", 150)])
+def test_single_plane_projections_report_their_accuracy(oracle, tree_name, n_prompt):
+    """MEDUSA_OPT_ACTIVATION_PLANES = 1: the projections read only the hi plane of every activation (half the tensor-core
+    work; four token tiles per weight stream).  This is an opt-in trade OUTSIDE the parity bar of the default path: the
+    inputs of every projection carry a bfloat16 rounding (2^-9 relative), and three layers deep the normalised hidden
+    state is off by 2.1e-2 .. 2.5e-2 instead of ~1e-2 -- just above the 2e-2 the default two-plane path is held to.  The
+    bound asserted here is the documented one of this mode (4e-2 hidden, 5e-2 logits); the measured values are printed."""
+    torch, B, U = _gpu()
+    spec = _spec(tree_name)
+    cfg = I.model_shape("tiny", d=512, n_heads=4, head_dim=128, ffn=1408, vocab=2048, n_medusa=4, n_layers=3,
+                        max_tree_nodes=spec["n_nodes"])
+    L_max = 512
+    w = I.make_weights(cfg, seed=3, dtype="bf16", gain_std=0.1)
+    ctx = U.make_ctx(cfg, "bf16", L_max, spec)
+    ctx.set_option(B.OPT_ACTIVATION_PLANES, 1)
+    ctx.load_weights(U.dev_weights(w))
+    om = oracle.Model(cfg, w, kv_bf16=True)
+    ot = oracle.build_tree_buffers(oracle.default_tree_paths(**spec))
+    prompt = I.make_prompt(n_prompt, cfg["vocab"], 4)
+    ctx.prefill(torch.from_numpy(prompt).cuda())
+    kc = np.zeros(om.cache_shape(L_max))
+    vc = np.zeros_like(kc)
+    L = 0
+    while L < n_prompt:
+        n = min(64, n_prompt - L)
+        last = oracle.tree_pass(om, prompt[L:L + n], oracle.chain_tree(n), L, kc, vc, want_logits=False)
+        oracle.accept_and_update_kv(last["tree_k"], last["tree_v"], kc, vc, np.arange(n), n - 1, n, L, last["hidden"], prompt[L:L + n])
+        L += n
+    T, d, V = ot["T"], cfg["d"], cfg["vocab"]
+    tok = I.rng(5, "treetok").integers(0, V, size=T).astype(np.int32)
+    ctx.tree_pass(torch.from_numpy(tok).cuda())
+    ref = oracle.tree_pass(om, tok, ot, n_prompt, kc, vc)
+    hid = ctx.read_workspace(B.WS_HIDDEN, (T, d), np.float32)
+    lgt = ctx.read_workspace(B.WS_LOGITS, (T, V), np.float32)
+    eh, el = np.abs(hid - ref["hidden"]).max(), np.abs(lgt - ref["logits"]).max()
+    print("single plane, %s: hidden max |err| %.3g, logits %.3g" % (tree_name, eh, el))
+    assert eh <= 2 * TOL_HIDDEN_BF16, "hidden max |err| %.3g" % eh
+    assert el <= TOL_LOGIT_BF16, "logits max |err| %.3g" % el
+    assert ctx.device_status() == 0
+    ctx.close()
