@@ -1137,11 +1137,12 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
     if (max_commit > depth1) max_commit = depth1;  // a step never commits more than one root-to-leaf path
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
 
-    // (no graphs while the tcgen05 attention kernel is forced into the step: it sizes its grid from the host's bound
-    // of the cache length, which a captured launch would freeze)
+    // (a captured launch of the tcgen05 attention kernel freezes the grid it sized from the host's bound of the cache
+    // length; the kernel copes with a cache that has grown past that bound -- its last grid row takes the remaining
+    // tiles -- so replaying it stays correct, only less evenly split)
     bool graphed = false;
     cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
-    if (c->step_graphs_on && !c->prof && c->skip_mask == 0 && c->attn_mode != 2 && c->withhold == 0 &&
+    if (c->step_graphs_on && !c->prof && c->skip_mask == 0 && c->withhold == 0 &&
         cudaStreamIsCapturing(c->stream, &capturing) == cudaSuccess && capturing == cudaStreamCaptureStatusNone) {
         medusa_ctx::StepKey key;
         memset(&key, 0, sizeof key);
