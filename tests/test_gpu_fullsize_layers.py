@@ -35,18 +35,25 @@ def _planes(ctx, B, which, rows, width):
     return (p[0].astype(np.float64) + p[1].astype(np.float64))[:rows]
 
 
-CASES = [("7b", 32, "sparse64_d4", (0, 15, 31)), ("13b", 40, "sparse64_d5", (0, 39)), ("7b", 1, "sparse64_d4", (0,)),
-         ("13b", 1, "sparse64_d5", (0,))]
+# the last field picks the attention kernel inside the pass: 0 the library's default, 2 the tcgen05 kernel forced.
+# The tcgen05 kernel takes the queries as one bfloat16 plane (tensor memory has no room for the residual plane), so
+# its rows are held to twice the flat bound on hidden states; it is opt-in inside a step for that reason.
+CASES = [("7b", 32, "sparse64_d4", (0, 15, 31), 0), ("13b", 40, "sparse64_d5", (0, 39), 0), ("7b", 1, "sparse64_d4", (0,), 0),
+         ("13b", 1, "sparse64_d5", (0,), 0), ("7b", 1, "sparse64_d4", (0,), 2), ("13b", 1, "sparse64_d5", (0,), 2)]
 
 
-@pytest.mark.parametrize("shape,n_layers,tree_name,tap_layers", CASES, ids=["%s_%dlayers" % (c[0], c[1]) for c in CASES])
-def test_every_row_of_a_layer_at_the_flat_tolerance(oracle, shape, n_layers, tree_name, tap_layers):
+@pytest.mark.parametrize("shape,n_layers,tree_name,tap_layers,attn_kernel", CASES,
+                         ids=["%s_%dlayers%s" % (c[0], c[1], "_tcgen05_attention" if c[4] == 2 else "") for c in CASES])
+def test_every_row_of_a_layer_at_the_flat_tolerance(oracle, shape, n_layers, tree_name, tap_layers, attn_kernel):
     torch, B, U = _gpu()
+    tol_hidden = TOL_HIDDEN_BF16 if attn_kernel == 0 else 2 * TOL_HIDDEN_BF16
     cfg = I.model_shape(shape, n_layers=n_layers)
     L_max, n_prompt = 4096, 520   # eight full prefill passes and a ragged one; the cache tiles end ragged too
     w = I.make_weights(cfg, seed=40, dtype="bf16")
     ctx = U.make_ctx(cfg, "bf16", L_max, I.TREE_SPECS[tree_name])
     ctx.load_weights(U.dev_weights(w))
+    if attn_kernel:
+        ctx.set_option(B.OPT_ATTENTION_KERNEL, attn_kernel)
     om = oracle.Model(cfg, w, kv_bf16=True)
     ot = oracle.build_tree_buffers(oracle.default_tree_paths(**I.TREE_SPECS[tree_name]))
     d, V, T = cfg["d"], cfg["vocab"], ot["T"]
@@ -81,8 +88,8 @@ def test_every_row_of_a_layer_at_the_flat_tolerance(oracle, shape, n_layers, tre
         # the residual stream itself, relative to its own scale (reported; the normalised form above is the criterion)
         e_x_rel = float(np.abs(x_out - ref["x_out"]).max() / np.sqrt(np.mean(ref["x_out"] ** 2)))
         report.append((l, e_att, e_xn, e_k, e_v, e_x_rel))
-        assert e_att <= TOL_HIDDEN_BF16, "layer %d: attention output max |err| %.3g on 64 rows" % (l, e_att)
-        assert e_xn <= TOL_HIDDEN_BF16, "layer %d: normalised hidden max |err| %.3g on 64 rows" % (l, e_xn)
+        assert e_att <= tol_hidden, "layer %d: attention output max |err| %.3g on 64 rows" % (l, e_att)
+        assert e_xn <= tol_hidden, "layer %d: normalised hidden max |err| %.3g on 64 rows" % (l, e_xn)
         assert e_k <= TOL_KV_BF16 and e_v <= TOL_KV_BF16, "layer %d: tree K/V max |err| %.3g / %.3g" % (l, e_k, e_v)
     # the closing stage on the GPU's own final hidden state: every logit of every row
     hid = ctx.read_workspace(B.WS_HIDDEN, (T, d), np.float32)
@@ -91,7 +98,7 @@ def test_every_row_of_a_layer_at_the_flat_tolerance(oracle, shape, n_layers, tre
     e_lg = float(np.abs(lg - lg_ref).max())
     assert e_lg <= TOL_LOGIT_BF16, "logits max |err| %.3g on 64 rows" % e_lg
     ctx.set_option(B.OPT_LAYER_TAP, -1)
-    line = "%s width, %d layers, all %d rows, L=%d: " % (shape, n_layers, T, n_prompt)
+    line = "%s width, %d layers, all %d rows, L=%d, attention kernel %d: " % (shape, n_layers, T, n_prompt, attn_kernel)
     line += "; ".join("layer %d att %.3g norm-hidden %.3g K %.3g V %.3g x(rel) %.3g" % r for r in report)
     line += "; logits on the GPU's hidden %.3g" % e_lg
     if n_layers == 1:
@@ -108,6 +115,6 @@ def test_every_row_of_a_layer_at_the_flat_tolerance(oracle, shape, n_layers, tre
         full = oracle.tree_pass(om, tok, ot, n_prompt, kc0, vc0)
         e_h, e_l = float(np.abs(hid - full["hidden"]).max()), float(np.abs(lg - full["logits"]).max())
         line += "; end to end vs the oracle's own pass: hidden %.3g logits %.3g" % (e_h, e_l)
-        assert e_h <= TOL_HIDDEN_BF16 and e_l <= TOL_LOGIT_BF16, line
+        assert e_h <= tol_hidden and e_l <= TOL_LOGIT_BF16, line
     print(line)
     ctx.close()
