@@ -22,6 +22,7 @@
  *   ora_tree_attention         Sec. 2.1.2, Fig. 2; App. G Table 5 ("parallel decoding" QK^T, PV)
  *   ora_tree_pass              App. G Table 5 (linears on q tokens) on a Llama-style block
  *   ora_evaluate_posterior     Sec. 2.3.1 (typical acceptance), Fig. 1 (longest accepted prefix)
+ *   ora_evaluate_rejection     Sec. 1 / Sec. 2.3.1 first paragraph (rejection sampling of speculative decoding, reused)
  *   ora_accept_and_update_kv   (paper silent; KV cache implied by Sec. 3.3 / App. G)
  *   ora_generate / ora_generate_plain   Sec. 2 (the three sub-steps per decoding step)
  *
@@ -854,6 +855,122 @@ void ora_evaluate_posterior(const float *logits, int32_t V, const int32_t *tree_
     }
     if (min_margin)
         *min_margin = mm;
+}
+
+/*
+ * Rejection-sampling acceptance (Sec. 1 and Sec. 2.3.1, first paragraph: the rejection sampling scheme of
+ * speculative decoding can be reused so that the output follows the original model's distribution).  The paper
+ * gives no algorithm for its candidate tree; the reading taken here is speculative sampling with the tree's
+ * candidates as DETERMINISTIC drafts (they are top-k picks, not samples, so a draft's proposal distribution is a
+ * point mass q = 1 on its token):
+ *   at node n with P = softmax(logits[n] / tau), its children c_1, c_2, ... in node order, R = 0:
+ *     child c_i with token x_i is accepted iff uniform[c_i] < P[x_i] / (1 - R)       (min(1, P/q) of the residual)
+ *     otherwise x_i is struck out, R += P[x_i], and the next sibling is tried against the renormalised residual;
+ *   an accepted child becomes n; when every child of n was rejected (or n is a leaf) the next token is drawn from
+ *   the residual of n: the Gumbel-max sample argmax_v fl32(fl32(logits[n][v] * inv_tau) + gumbel[v]) over the
+ *   tokens v that were not struck out at n (ties -> lower index).
+ * Each emitted token then has exactly the backbone's sampling distribution: P(x_i emitted) =
+ * prod_{j<i} (1 - a_j) * a_i = P[x_i], and a token outside the children keeps its mass P[v].
+ * uniform: [T] numbers in [0, 1), one per node (the entry of a node is used when that node is tried).
+ * Outputs as ora_evaluate_posterior; best = the lowest retrieve row that starts with the accepted path;
+ * rejected_tok (nullable, [T]) / n_rejected: the tokens struck out at the last node;
+ * min_margin (nullable): smallest |u - a| / a over the decisions taken.  Requires tau > 0.
+ */
+void ora_evaluate_rejection(const float *logits, int32_t V, const int32_t *tree_tok, const int32_t *parent, int32_t T,
+                            const int32_t *retrieve, int32_t P, int32_t depth, double tau, const float *gumbel,
+                            const float *uniform, int32_t *best, int32_t *accept_len, int32_t *next_root,
+                            int32_t *acc_nodes, int32_t *rejected_tok, int32_t *n_rejected, double *min_margin)
+{
+    int W = depth + 1;
+    int n = 0, len = 0, nrej = 0;
+    double mm = INFINITY;
+    int32_t *rej = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T > 0 ? T : 1));
+    acc_nodes[0] = 0;
+    for (;;) {
+        const float *lp = logits + (size_t)n * V;
+        double mx = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+            double l = (double)lp[v] / tau;
+            if (l > mx)
+                mx = l;
+        }
+        double se = 0.0;
+        for (int v = 0; v < V; ++v)
+            se += exp((double)lp[v] / tau - mx);
+        double lse = mx + log(se);
+        double R = 0.0;
+        int accepted = -1;
+        nrej = 0;
+        for (int c = 0; c < T; ++c) {
+            if (c == n || parent[c] != n)
+                continue;
+            double pc = exp((double)lp[tree_tok[c]] / tau - lse);
+            double rem = 1.0 - R;
+            double a = rem > 0.0 ? pc / rem : 1.0;
+            double u = (double)uniform[c];
+            if (a > 0.0) {
+                double mg = fabs(u - a) / a;
+                if (mg < mm)
+                    mm = mg;
+            }
+            if (u < a) {
+                accepted = c;
+                break;
+            }
+            R += pc;
+            rej[nrej++] = tree_tok[c];
+        }
+        if (accepted < 0)
+            break;
+        n = accepted; /* a tree of this depth has no node deeper than W - 1, so len stays below W */
+        acc_nodes[++len] = n;
+    }
+    for (int j = len + 1; j < W; ++j)
+        acc_nodes[j] = -1;
+    *accept_len = len;
+    int b = 0;
+    for (int r = 0; r < P; ++r) {
+        int same = 1;
+        for (int j = 0; j <= len; ++j)
+            if (retrieve[(size_t)r * W + j] != acc_nodes[j]) {
+                same = 0;
+                break;
+            }
+        if (same) {
+            b = r;
+            break;
+        }
+    }
+    *best = b;
+    {
+        const float *ll = logits + (size_t)n * V;
+        float inv_tau = (float)(1.0 / tau);
+        int bi = -1;
+        float bs = 0.f;
+        for (int v = 0; v < V; ++v) {
+            int struck = 0;
+            for (int q = 0; q < nrej; ++q)
+                if (rej[q] == v)
+                    struck = 1;
+            if (struck)
+                continue;
+            volatile float sc = ll[v] * inv_tau; /* one rounding per operation, no fused multiply-add */
+            volatile float s = sc + gumbel[v];
+            if (bi < 0 || s > bs) {
+                bs = s;
+                bi = v;
+            }
+        }
+        *next_root = bi < 0 ? 0 : bi;
+    }
+    if (rejected_tok)
+        for (int q = 0; q < nrej; ++q)
+            rejected_tok[q] = rej[q];
+    if (n_rejected)
+        *n_rejected = nrej;
+    if (min_margin)
+        *min_margin = mm;
+    free(rej);
 }
 
 /*

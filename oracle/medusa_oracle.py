@@ -315,16 +315,34 @@ def final_norm_lm_head(model: Model, x=None, hidden_in=None, want_logits=True):
 
 # ----------------------------------------------------------------------------- acceptance / commit
 
-GREEDY, TYPICAL = 0, 1
+GREEDY, TYPICAL, REJECTION = 0, 1, 2
 
 
-def evaluate_posterior(logits_f32, tree_tok, tree, mode=GREEDY, tau=0.0, eps=0.09, delta=0.3, gumbel=None):
+def evaluate_posterior(logits_f32, tree_tok, tree, mode=GREEDY, tau=0.0, eps=0.09, delta=0.3, gumbel=None, uniform=None):
+    """Acceptance of one step.  mode REJECTION (needs tau > 0, gumbel [V] and uniform [T]) also returns `rejected`, the
+    tokens struck out at the last accepted node."""
     lg = _f32(logits_f32)
     T, V = lg.shape
     tok = _i32(tree_tok)
     if tok.size and (tok.min() < 0 or tok.max() >= V):
         raise ValueError("tree token outside the vocabulary [0, %d)" % V)
     W = tree["depth"] + 1
+    if mode == REJECTION:
+        if not tau > 0.0 or gumbel is None or uniform is None:
+            raise ValueError("rejection sampling needs a temperature above zero, a Gumbel row and one uniform per node")
+        g, u = _f32(gumbel), _f32(uniform)
+        if g.size != V or u.size != tree["T"]:
+            raise ValueError("gumbel must have V entries and uniform T")
+        best, alen, nroot, nrej, margin = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32(), C.c_double()
+        acc = np.full(W, -1, dtype=np.int32)
+        rej = np.full(tree["T"], -1, dtype=np.int32)
+        par, ret = _i32(tree["parent"]), _i32(tree["retrieve"])
+        lib().ora_evaluate_rejection(_p(lg), C.c_int32(V), _p(tok), _p(par), C.c_int32(tree["T"]),
+                                     _p(ret), C.c_int32(tree["P"]), C.c_int32(tree["depth"]),
+                                     C.c_double(tau), _p(g), _p(u), C.byref(best), C.byref(alen), C.byref(nroot), _p(acc),
+                                     _p(rej), C.byref(nrej), C.byref(margin))
+        return dict(best=best.value, accept_len=alen.value, next_root=nroot.value, acc_nodes=acc,
+                    min_margin=margin.value, rejected=rej[:nrej.value].copy())
     best = C.c_int32()
     alen = C.c_int32()
     nroot = C.c_int32()

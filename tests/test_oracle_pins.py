@@ -737,3 +737,187 @@ def test_large_tree_medusa_greedy_equals_plain_greedy(oracle):
     plain = oracle.generate_plain(om, prompt, G, 64)
     assert ref["tokens"].tolist() == plain["tokens"].tolist()
     assert ref["emitted_per_step"].sum() == G and ref["emitted_per_step"].max() <= t["depth"] + 1
+
+
+# ----------------------------------------------------------------------------- rejection sampling (Sec. 1, Sec. 2.3.1 first paragraph)
+
+def _flat_tree(oracle, n_children):
+    """Root with n_children leaf children (nodes 1..n in rank order)."""
+    return oracle.build_tree_buffers(np.array([[i] for i in range(n_children)], dtype=np.int32))
+
+
+def _accept_probability(oracle, logits, tok, t, tau, child, reject_before):
+    """The probability with which the oracle accepts node `child`, read off its decisions: the uniform at which the
+    decision flips (bisection in float32), with every node of `reject_before` forced to be rejected first."""
+    V = logits.shape[1]
+    zero = np.zeros(V, dtype=np.float32)
+    lo, hi = np.float32(0.0), np.float32(1.0)
+    for _ in range(40):
+        mid = np.float32((np.float64(lo) + np.float64(hi)) / 2)
+        u = np.zeros(t["T"], dtype=np.float32)
+        u[list(reject_before)] = np.float32(0.99999994)
+        u[child] = mid
+        r = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=tau, gumbel=zero, uniform=u)
+        if child in r["acc_nodes"].tolist():
+            lo = mid
+        else:
+            hi = mid
+    return float(hi)
+
+
+def test_rejection_sampling_hand_vectors(oracle):
+    fx = json.load(open(os.path.join(GOLD, "rejection_sampling_vectors.json")))["cases"]
+    for c in fx:
+        lg = np.array(c["logits"], dtype=np.float32)
+        V, m = lg.size, len(c["children_tokens"])
+        t = _flat_tree(oracle, m)
+        tok = np.array([0] + c["children_tokens"], dtype=np.int32)
+        logits = np.tile(lg, (t["T"], 1))
+        assert abs(sum(c["p"]) - 1.0) < 5e-6
+        # the acceptance probability of every sibling, as the oracle takes its decisions, against the hand values
+        for i in range(m):
+            a = _accept_probability(oracle, logits, tok, t, c["tau"], 1 + i, range(1, 1 + i))
+            assert abs(a - c["accept_prob"][i]) < 3e-6, (c["children_tokens"], i, a)
+        for tr in c["trials"]:
+            u = np.array([0.0] + tr["uniform"], dtype=np.float32)
+            r = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=c["tau"], gumbel=np.zeros(V, np.float32),
+                                          uniform=u)
+            k = tr["accepted_child"]
+            if k >= 0:
+                assert r["accept_len"] == 1 and r["acc_nodes"].tolist() == [0, 1 + k], (tr, r)
+                assert r["rejected"].tolist() == [] and r["best"] == k
+                if tr.get("decides_by_renormalisation"):
+                    x = c["children_tokens"][k]
+                    assert c["p"][x] < tr["uniform"][k] < c["accept_prob"][k]
+            else:
+                assert r["accept_len"] == 0 and r["acc_nodes"].tolist() == [0, -1]
+                assert sorted(r["rejected"].tolist()) == sorted(c["children_tokens"])
+                # the next token comes from the residual: never a rejected token, frequencies as worked by hand
+                noise = I.gumbel_noise(6000, V, 77)
+                counts = np.zeros(V)
+                for row in noise:
+                    counts[oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=c["tau"], gumbel=row,
+                                                     uniform=u)["next_root"]] += 1
+                for x in c["children_tokens"]:
+                    assert counts[x] == 0
+                for key, q in tr["residual"].items():
+                    f = counts[int(key)] / len(noise)
+                    assert abs(f - q) < 4 * math.sqrt(max(q * (1 - q), 1e-4) / len(noise)) + 1e-9, (key, f, q)
+
+
+def test_rejection_sampling_keeps_the_backbone_distribution(oracle):
+    """Losslessness, the property the scheme is for: the probability that the step's first new token is x equals
+    softmax(logits / tau)[x].  For a child x_i that probability is prod_{j<i}(1 - a_j) * a_i with the oracle's own
+    acceptance probabilities a (read off its decisions); a wrong renormalisation, sibling order or temperature breaks it."""
+    g = I.rng(31, "rej")
+    V, m, tau = 12, 5, 0.8
+    t = _flat_tree(oracle, m)
+    lg = (g.standard_normal(V) * 2.0).astype(np.float32)
+    logits = np.tile(lg, (t["T"], 1))
+    tok = np.concatenate([[0], g.permutation(V)[:m]]).astype(np.int32)
+    x = lg.astype(np.float64) / tau
+    p = np.exp(x - x.max())
+    p /= p.sum()
+    reach = 1.0
+    for i in range(m):
+        a = _accept_probability(oracle, logits, tok, t, tau, 1 + i, range(1, 1 + i))
+        assert abs(reach * a - p[tok[1 + i]]) < 2e-6, (i, reach * a, p[tok[1 + i]])
+        reach *= 1.0 - a
+    # what is left is the mass of the tokens that are no child, and the residual sample lands only there
+    rest = [v for v in range(V) if v not in tok[1:].tolist()]
+    assert abs(reach - p[rest].sum()) < 5e-6
+    u = np.full(t["T"], 0.99999994, dtype=np.float32)
+    noise = I.gumbel_noise(8000, V, 78)
+    counts = np.zeros(V)
+    for row in noise:
+        r = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=tau, gumbel=row, uniform=u)
+        assert r["accept_len"] == 0
+        counts[r["next_root"]] += 1
+    assert counts[tok[1:]].sum() == 0
+    for v in rest:
+        q = p[v] / p[rest].sum()
+        assert abs(counts[v] / len(noise) - q) < 4 * math.sqrt(max(q * (1 - q), 1e-4) / len(noise)), (v, counts[v] / len(noise), q)
+
+
+def test_rejection_sampling_walks_the_tree_with_each_nodes_own_logits(oracle):
+    g = I.rng(32, "rejtree")
+    spec = I.TREE_SPECS["sparse64_d4"]
+    t = oracle.build_tree_buffers(oracle.default_tree_paths(**spec))
+    T, V, W = t["T"], 50, t["depth"] + 1
+    logits = g.standard_normal((T, V)).astype(np.float32)
+    tok = np.zeros(T, dtype=np.int32)
+    for n in range(T):  # siblings carry distinct tokens, as top-k picks do
+        kids = [c for c in range(T) if c != n and t["parent"][c] == n]
+        tok[kids] = g.permutation(V)[:len(kids)]
+    zero = np.zeros(V, dtype=np.float32)
+    # uniforms of zero accept the first child everywhere: the all-rank-0 path, full depth, next token from the leaf's row
+    r = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=1.0, gumbel=zero, uniform=np.zeros(T, np.float32))
+    assert r["accept_len"] == t["depth"] and r["acc_nodes"].tolist() == t["retrieve"][r["best"]][:W].tolist()
+    assert all(t["parent"][r["acc_nodes"][j]] == r["acc_nodes"][j - 1] for j in range(1, W))
+    assert r["next_root"] == int(np.argmax(logits[r["acc_nodes"][-1]]))
+    # uniforms just below one reject everything: nothing accepted, the children's tokens struck out at the root
+    r = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=1.0, gumbel=zero,
+                                  uniform=np.full(T, 0.99999994, np.float32))
+    kids0 = [c for c in range(T) if c != 0 and t["parent"][c] == 0]
+    assert r["accept_len"] == 0 and r["rejected"].tolist() == tok[kids0].tolist()
+    masked = logits[0].copy()
+    masked[tok[kids0]] = -np.inf
+    assert r["next_root"] == int(np.argmax(masked))
+    # brute force of the definition, node by node, on random uniforms
+    for trial in range(20):
+        u = g.random(T).astype(np.float32)
+        noise = I.gumbel_noise(1, V, 100 + trial)[0]
+        r = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=0.9, gumbel=noise, uniform=u)
+        n, path, struck = 0, [0], []
+        while True:
+            x = logits[n].astype(np.float64) / 0.9
+            p = np.exp(x - x.max())
+            p /= p.sum()
+            R, nxt, struck = 0.0, -1, []
+            for c in range(T):
+                if c != n and t["parent"][c] == n:
+                    if float(u[c]) < p[tok[c]] / (1.0 - R):
+                        nxt = c
+                        break
+                    R += p[tok[c]]
+                    struck.append(int(tok[c]))
+            if nxt < 0:
+                break
+            n = nxt
+            path.append(n)
+        assert r["acc_nodes"][:len(path)].tolist() == path and r["accept_len"] == len(path) - 1
+        assert r["rejected"].tolist() == struck
+        assert t["retrieve"][r["best"]][:len(path)].tolist() == path
+        sc = (logits[n] * np.float32(1.0 / 0.9)).astype(np.float32) + noise
+        sc[struck] = -np.inf
+        assert r["next_root"] == int(np.argmax(sc))
+        assert r["min_margin"] > 0.0
+
+
+def test_rejection_sampling_at_low_temperature_is_greedy(oracle):
+    g = I.rng(33, "rejcold")
+    spec = I.TREE_SPECS["sparse64_d4"]
+    t = oracle.build_tree_buffers(oracle.default_tree_paths(**spec))
+    T, V = t["T"], 40
+    for trial in range(6):
+        logits = g.standard_normal((T, V)).astype(np.float32)
+        tok = g.integers(0, V, size=T).astype(np.int32)
+        # plant the argmax token on a path so that greedy acceptance has something to accept
+        row = t["retrieve"][trial % t["P"]]
+        for j in range(1, t["depth"] + 1):
+            if row[j] >= 0 and j <= 1 + trial % 3:
+                tok[row[j]] = int(np.argmax(logits[row[j - 1]]))
+        for n in range(T):  # keep siblings distinct without touching planted nodes
+            kids = [c for c in range(T) if c != n and t["parent"][c] == n]
+            seen = set()
+            for c in kids:
+                while int(tok[c]) in seen:
+                    tok[c] = (tok[c] + 1) % V if c not in row else tok[c]
+                    if c in row:
+                        break
+                seen.add(int(tok[c]))
+        gr = oracle.evaluate_posterior(logits, tok, t, mode=oracle.GREEDY)
+        u = g.random(T).astype(np.float32) * np.float32(0.98) + np.float32(0.01)
+        rj = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=1e-3, gumbel=np.zeros(V, np.float32), uniform=u)
+        assert rj["accept_len"] == gr["accept_len"] and rj["next_root"] == gr["next_root"]
+        assert rj["acc_nodes"].tolist() == gr["acc_nodes"].tolist()
