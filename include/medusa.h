@@ -42,7 +42,7 @@ enum {
 };
 
 enum { MEDUSA_F32 = 0, MEDUSA_BF16 = 1 };
-enum { MEDUSA_GREEDY = 0, MEDUSA_TYPICAL = 1 };
+enum { MEDUSA_GREEDY = 0, MEDUSA_TYPICAL = 1, MEDUSA_REJECTION = 2 };
 
 /* Llama-style decoder shape (paper App. G names the operators: QKV/O linears, QK^T/PV, up/gate/down). */
 typedef struct {
@@ -76,7 +76,15 @@ typedef struct {
 } medusa_tree_buffers;
 
 /* Acceptance rule (paper Sec. 2.3.1).  temperature <= 0 or mode GREEDY: accept a child iff it is the
- * argmax of its parent's logits.  TYPICAL: iff p > min(eps, delta*exp(-H(p))), p = softmax(logits/temperature). */
+ * argmax of its parent's logits.  TYPICAL: iff p > min(eps, delta*exp(-H(p))), p = softmax(logits/temperature).
+ * REJECTION (paper Sec. 1 and Sec. 2.3.1, first paragraph: the rejection sampling of speculative decoding, which keeps
+ * the original model's distribution; the paper gives no algorithm for the tree, this is the reading taken): the tree's
+ * candidates are deterministic drafts (point-mass proposals).  Starting at the root, the children of the current node
+ * are tried in node order: child c with token x is accepted iff uniform[c] < p(x) / (1 - R), R = the mass of the
+ * siblings rejected before it at this node; an accepted child becomes the current node; when all children are
+ * rejected (or the node is a leaf) the next token is the Gumbel-max sample of the node's distribution without the
+ * rejected tokens.  Needs temperature > 0 and a noise row of V + T floats: gumbel[V] followed by uniform[T] in [0, 1)
+ * (eps and delta are ignored).  Decisions are taken in double precision. */
 typedef struct {
     int32_t mode;
     float temperature, eps, delta;
@@ -269,7 +277,9 @@ int32_t medusa_tree_attention_static(const void *q, const void *k_new, const voi
  * Outputs (device): best (row), accept_len (speculated tokens accepted, 0..depth), acc_nodes [depth+1]
  * (-1 beyond accept_len), next_root = argmax logits[last accepted node] (ties: lower index), or, if
  * gumbel != NULL and TYPICAL with temperature > 0, argmax_v fl(fl(logit_v * fl(1/temperature)) + gumbel[v]).
- * Typical-mode statistics are evaluated in double precision. */
+ * Typical-mode statistics are evaluated in double precision.  REJECTION: gumbel holds V + T floats (see
+ * medusa_accept_params), best = the lowest retrieve row that starts with the accepted path; INVALID_ARG without a
+ * noise row or with temperature <= 0. */
 int32_t medusa_evaluate_posterior(medusa_ctx *ctx, const float *logits, const int32_t *tree_tok,
                                   const medusa_accept_params *params, const float *gumbel, int32_t *best,
                                   int32_t *accept_len, int32_t *next_root, int32_t *acc_nodes);
@@ -301,7 +311,8 @@ int32_t medusa_prefill(medusa_ctx *ctx, const int32_t *prompt, int32_t n);
  * mask/positions against the context's cache; results stay in the workspace (LOGITS, HIDDEN, TREE_K/V). */
 int32_t medusa_tree_pass(medusa_ctx *ctx, const int32_t *tokens);
 /* One full step: heads on h_last -> top-k -> tree tokens -> tree pass -> acceptance -> commit.
- * max_commit clamps the tokens emitted (generation budget).  gumbel (nullable): float [V] noise for this step.
+ * max_commit clamps the tokens emitted (generation budget).  gumbel (nullable): float [V] noise for this step
+ * (REJECTION: required, float [V + T]).
  * emitted_host / n_emitted_host (nullable, pinned host memory recommended): async copies of the emitted
  * tokens [depth+1] and their count, valid after the stream is synchronised.
  * Nothing is synchronised: the step is enqueued on the context's stream.  The second consecutive step with the
@@ -323,7 +334,7 @@ int32_t medusa_select_sequence(medusa_ctx *ctx, int32_t b);
  * pass (LOGITS, HIDDEN, TREE_K/V, TREE_TOK use the same rows), the projections stream the weights once for all sequences,
  * the attention runs per sequence against that sequence's cache and cache length, and heads, top-k, acceptance and
  * commit run per sequence exactly as in medusa_decode_step (same acceptance rule for all).  The uploaded tree must have
- * at most 64 nodes (SHAPE otherwise).  gumbel (nullable): float [B][V] device noise rows; emitted_host [B][depth+1] and
+ * at most 64 nodes (SHAPE otherwise).  gumbel (nullable): float [B][V] device noise rows ([B][V + T] for REJECTION); emitted_host [B][depth+1] and
  * n_emitted_host [B] (nullable, pinned host memory recommended): async copies, valid after the stream is synchronised.
  * Every sequence must have been prefilled.  The step is enqueued directly (no whole-step graph). */
 int32_t medusa_decode_step_batch(medusa_ctx *ctx, const medusa_accept_params *params, const float *gumbel,
@@ -331,7 +342,7 @@ int32_t medusa_decode_step_batch(medusa_ctx *ctx, const medusa_accept_params *pa
 
 /* Convenience loop with HOST buffers: prefill prompt_host[n_prompt], then decode steps until G tokens are
  * emitted (one stream synchronisation per step to read the emitted tokens).  gumbel_host (nullable):
- * [max steps = G][V].  Writes out_tokens_host[G]; emitted_per_step_host (nullable) [G]; *steps_host. */
+ * [max steps = G][V] ([G][V + T] for REJECTION, where it is required).  Writes out_tokens_host[G]; emitted_per_step_host (nullable) [G]; *steps_host. */
 int32_t medusa_generate(medusa_ctx *ctx, const int32_t *prompt_host, int32_t n_prompt, int32_t G,
                         const medusa_accept_params *params, const float *gumbel_host, int32_t *out_tokens_host,
                         int32_t *emitted_per_step_host, int32_t *steps_host);

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_PKG, "libmedusa_b200.so")
 
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_CACHE_FULL, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6, -7
 F32, BF16 = 0, 1
-GREEDY, TYPICAL = 0, 1
+GREEDY, TYPICAL, REJECTION = 0, 1, 2  # REJECTION: the noise row is gumbel[V] followed by uniform[T]
 (WS_LOGITS, WS_HIDDEN, WS_TREE_K, WS_TREE_V, WS_K_CACHE, WS_V_CACHE, WS_HEAD_LOGITS, WS_TOPK_IDX, WS_TREE_TOK,
  WS_ACC_NODES, WS_STATE, WS_H_LAST, WS_EMITTED, WS_TAP_X_IN, WS_TAP_X_OUT, WS_TAP_ATT, WS_TAP_XN_OUT) = range(17)
 (OPT_STEP_GRAPHS, OPT_ATTENTION_KERNEL, OPT_ATTENTION_LENGTH_HINT, OPT_LAYER_TAP, OPT_SPIN_LIMIT,

@@ -453,7 +453,7 @@ static void point_at(medusa_ctx *c, int b)
     c->topk_idx = c->topk_idx_all + (size_t)b * K * R;
     c->acc_nodes = c->acc_nodes_all + (size_t)b * TREE_ROWS;
     c->emitted = c->emitted_all + (size_t)b * TREE_ROWS;
-    c->gumbel_dev = c->gumbel_all + (size_t)b * m.vocab;
+    c->gumbel_dev = c->gumbel_all + (size_t)b * ((size_t)m.vocab + c->rows);
     c->k_cache = c->k_cache_all ? c->k_cache_all + (size_t)b * c->cache_seq_bytes : nullptr;
     c->v_cache = c->v_cache_all ? c->v_cache_all + (size_t)b * c->cache_seq_bytes : nullptr;
     if ((size_t)b < c->L_upper_all.size()) c->L_upper = c->L_upper_all[b];
@@ -538,7 +538,7 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     TRY(dev_alloc(c, &c->node_lse, R));
     TRY(dev_alloc(c, &c->node_ent, R));
     TRY(dev_alloc_bytes(c, &c->node_part, R * NODE_STAT_SLICES * NODE_PART_BYTES));
-    TRY(dev_alloc(c, &c->gumbel_all, NB * V));
+    TRY(dev_alloc(c, &c->gumbel_all, NB * (V + R)));  // per sequence: Gumbel noise [V], then one uniform per token row
     point_at(c, 0);
     TRY(dev_alloc_bytes(c, &c->topk_scratch, topk_scratch_bytes(m.n_medusa > 0 ? m.n_medusa : 1)));
     TRY(dev_alloc(c, &c->tap_x_in, R * d));
@@ -888,6 +888,15 @@ extern "C" int32_t medusa_tree_attention(medusa_ctx *c, const void *q, const voi
 
 // ============================================================================ a7: acceptance
 
+static bool known_mode(int32_t mode) { return mode == MEDUSA_GREEDY || mode == MEDUSA_TYPICAL || mode == MEDUSA_REJECTION; }
+// floats of one step's noise row: Gumbel noise for the vocabulary, for rejection sampling also one uniform per tree node
+static size_t noise_floats(const medusa_ctx *c, int32_t mode)
+{
+    return (size_t)c->m.vocab + (mode == MEDUSA_REJECTION ? (size_t)c->tree.T : 0);
+}
+// whether the acceptance kernels read the noise row in this mode
+static bool mode_reads_noise(const medusa_accept_params *p) { return p->mode == MEDUSA_TYPICAL || p->mode == MEDUSA_REJECTION; }
+
 extern "C" int32_t medusa_evaluate_posterior(medusa_ctx *c, const float *logits, const int32_t *tree_tok,
                                              const medusa_accept_params *params, const float *gumbel, int32_t *best,
                                              int32_t *accept_len, int32_t *next_root, int32_t *acc_nodes)
@@ -895,11 +904,14 @@ extern "C" int32_t medusa_evaluate_posterior(medusa_ctx *c, const float *logits,
     TRY(check_ready(c, true, false));
     if (!logits || !tree_tok || !params || !best || !accept_len || !next_root || !acc_nodes)
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_evaluate_posterior: null pointer");
-    if (params->mode != MEDUSA_GREEDY && params->mode != MEDUSA_TYPICAL)
+    if (!known_mode(params->mode))
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_evaluate_posterior: unknown mode %d", params->mode);
+    if (params->mode == MEDUSA_REJECTION && (!gumbel || !(params->temperature > 0.f)))
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_evaluate_posterior: rejection sampling needs a noise row and a temperature above zero");
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
     PosteriorArgs a{};
     a.logits = logits; a.tree_tok = tree_tok; a.retrieve = c->d_retrieve; a.parent = c->d_parent; a.gumbel = gumbel;
+    a.uniform = params->mode == MEDUSA_REJECTION ? gumbel + c->m.vocab : nullptr;  // the noise row is gumbel[V], uniform[T]
     a.T = c->tree.T; a.V = c->m.vocab; a.P = c->tree.P; a.depth = c->tree.depth; a.mode = params->mode;
     a.temperature = params->temperature; a.eps = params->eps; a.delta = params->delta;
     a.node_argmax = c->node_argmax; a.node_lse = c->node_lse; a.node_ent = c->node_ent;
@@ -1130,8 +1142,10 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
     TRY(check_ready(c, true, true));
     if (!params) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step: null params");
     if (max_commit < 1) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step: max_commit must be >= 1");
-    if (params->mode != MEDUSA_GREEDY && params->mode != MEDUSA_TYPICAL)
+    if (!known_mode(params->mode))
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step: unknown mode %d", params->mode);
+    if (params->mode == MEDUSA_REJECTION && (!gumbel || !(params->temperature > 0.f)))
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step: rejection sampling needs a noise row and a temperature above zero");
     const medusa_model_desc &m = c->m;
     const int32_t depth1 = c->tree.depth + 1;
     if (max_commit > depth1) max_commit = depth1;  // a step never commits more than one root-to-leaf path
@@ -1148,7 +1162,7 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
         memset(&key, 0, sizeof key);
         key.max_commit = max_commit;
         key.seq = c->cur;
-        const bool noisy = gumbel && params->mode == MEDUSA_TYPICAL;  // the acceptance kernel's own condition
+        const bool noisy = gumbel && mode_reads_noise(params);  // the acceptance kernel's own condition
         key.has_gumbel = noisy ? 1 : 0;
         key.p = *params;
         key.emitted_host = emitted_host;
@@ -1165,7 +1179,7 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
         if (g) {
             // the graph reads the step's noise row from the context's own buffer
             if (noisy && gumbel != c->gumbel_dev)
-                MEDUSA_CUDA(c, cudaMemcpyAsync(c->gumbel_dev, gumbel, (size_t)m.vocab * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->gumbel_dev, gumbel, noise_floats(c, params->mode) * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
             MEDUSA_CUDA(c, cudaGraphLaunch(g->exec, c->stream));
             for (int i = 0; i < MEDUSA_PROF_CATEGORIES; ++i) c->launches[i] += g->launches[i];
             g->used = ++c->step_clock;
@@ -1197,8 +1211,10 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
     TRY(check_ready(c, true, true));
     if (!params) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: null params");
     if (max_commit < 1) return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: max_commit must be >= 1");
-    if (params->mode != MEDUSA_GREEDY && params->mode != MEDUSA_TYPICAL)
+    if (!known_mode(params->mode))
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: unknown mode %d", params->mode);
+    if (params->mode == MEDUSA_REJECTION && (!gumbel || !(params->temperature > 0.f)))
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_decode_step_batch: rejection sampling needs noise rows and a temperature above zero");
     if (c->tree.T > TREE_ROWS)
         return fail(c, MEDUSA_ERR_SHAPE, "a batched step gives every sequence one tile of 64 token rows: the tree has %d nodes", c->tree.T);
     const medusa_model_desc &m = c->m;
@@ -1241,7 +1257,7 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
         int32_t *st = c->d_state;
         const size_t ro = (size_t)b * TREE_ROWS;
         rc = medusa_evaluate_posterior(c, c->logits + ro * m.vocab, c->tree_tok + ro, params,
-                                       gumbel ? gumbel + (size_t)b * m.vocab : nullptr, st + ST_BEST, st + ST_ACCEPT_LEN,
+                                       gumbel ? gumbel + (size_t)b * noise_floats(c, params->mode) : nullptr, st + ST_BEST, st + ST_ACCEPT_LEN,
                                        st + ST_NEXT_ROOT, c->acc_nodes);
         if (rc != MEDUSA_OK) break;
         CommitArgs a{};
@@ -1287,12 +1303,15 @@ extern "C" int32_t medusa_generate(medusa_ctx *c, const int32_t *prompt_host, in
     cudaFree(pd);
     if (rc != MEDUSA_OK) return rc;
     int32_t L = n_prompt, n_out = 0, steps = 0;
-    const bool sample = gumbel_host && params->mode == MEDUSA_TYPICAL && params->temperature > 0.f;
+    if (!known_mode(params->mode) || (params->mode == MEDUSA_REJECTION && (!gumbel_host || !(params->temperature > 0.f))))
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_generate: unknown mode, or rejection sampling without noise rows or with temperature <= 0");
+    const bool sample = gumbel_host && mode_reads_noise(params) && params->temperature > 0.f;
+    const size_t nf = noise_floats(c, params->mode);
     while (n_out < G) {
         int32_t budget = G - n_out < m.L_max - L ? G - n_out : m.L_max - L;
         if (budget <= 0) break;
         if (sample)
-            MEDUSA_CUDA(c, cudaMemcpyAsync(c->gumbel_dev, gumbel_host + (size_t)steps * m.vocab, (size_t)m.vocab * sizeof(float),
+            MEDUSA_CUDA(c, cudaMemcpyAsync(c->gumbel_dev, gumbel_host + (size_t)steps * nf, nf * sizeof(float),
                                            cudaMemcpyHostToDevice, c->stream));
         TRY(medusa_decode_step(c, params, sample ? c->gumbel_dev : nullptr, budget, c->pinned, c->pinned + TREE_ROWS));
         MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));

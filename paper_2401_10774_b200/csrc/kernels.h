@@ -102,6 +102,7 @@ struct PosteriorArgs {
     const int32_t *retrieve;  // [P][depth+1]
     const int32_t *parent;    // [T]
     const float *gumbel;      // nullable [V]
+    const float *uniform;     // [T] numbers in [0, 1): rejection sampling only
     int T, V, P, depth, mode;
     float temperature, eps, delta;
     // scratch

@@ -151,15 +151,22 @@ node_stats_kernel(const float *__restrict__ logits, int V, int typical, double t
     }
 }
 
-// one block: thread r walks retrieve row r; thread 0 picks the longest (lowest row on ties)
+// one block: thread r walks retrieve row r; thread 0 picks the longest (lowest row on ties).
+// rejection != 0 (rejection sampling with the candidates as deterministic drafts; needs the typical statistics):
+// the block walks down from the root instead -- per level every thread evaluates p of "its" node if that node is a
+// child of the current one, thread 0 tries the children in node order against the renormalised residual -- and the
+// next token is the Gumbel-max sample over the tokens that were not rejected at the last node.
 __global__ void __launch_bounds__(256)
-select_path_kernel(PosteriorArgs a, int typical, double tau, double eps, double delta)
+select_path_kernel(PosteriorArgs a, int typical, double tau, double eps, double delta, int rejection)
 {
     pdl_enter();
     __shared__ int s_len[MAX_T];
     __shared__ float sv[32];
     __shared__ int si[32];
     __shared__ int s_last;
+    __shared__ double s_pc[MAX_T];
+    __shared__ int s_rej[MAX_T];
+    __shared__ int s_nrej, s_cur, s_stop;
     const int W = a.depth + 1;
     const int r = threadIdx.x;
     if (typical && threadIdx.x < a.T) {
@@ -186,6 +193,94 @@ select_path_kernel(PosteriorArgs a, int typical, double tau, double eps, double 
     }
     if (typical)
         __syncthreads();  // the statistics written above are read by other threads of this (only) block
+    if (rejection) {
+        const int W1 = a.depth + 1;
+        if (threadIdx.x == 0) {
+            s_cur = 0;
+            s_stop = 0;
+            s_nrej = 0;
+            a.acc_nodes[0] = 0;
+            *a.accept_len = 0;
+        }
+        __syncthreads();
+        int len = 0;  // kept by every thread: all of them see the same s_cur / s_stop
+        for (int lvl = 0; lvl < W1; ++lvl) {
+            const int n = s_cur;
+            if (threadIdx.x < a.T) {
+                const int cnode = threadIdx.x;
+                s_pc[cnode] = cnode != n && a.parent[cnode] == n
+                                  ? exp((double)a.logits[(size_t)n * a.V + a.tree_tok[cnode]] / tau - a.node_lse[n])
+                                  : -1.0;  // not a child of the current node
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                double R = 0.0;
+                int accepted = -1, nrej = 0;
+                for (int cnode = 0; cnode < a.T; ++cnode) {
+                    const double pc = s_pc[cnode];
+                    if (pc < 0.0)
+                        continue;
+                    const double rem = 1.0 - R;
+                    const double acc_p = rem > 0.0 ? pc / rem : 1.0;
+                    if ((double)a.uniform[cnode] < acc_p) {
+                        accepted = cnode;
+                        break;
+                    }
+                    R += pc;
+                    s_rej[nrej++] = a.tree_tok[cnode];
+                }
+                s_nrej = nrej;
+                if (accepted < 0 || len + 1 >= W1) {
+                    s_stop = 1;
+                } else {
+                    s_cur = accepted;
+                    a.acc_nodes[len + 1] = accepted;
+                }
+            }
+            __syncthreads();
+            if (s_stop)
+                break;
+            ++len;
+        }
+        const int last_node = s_cur, nrej = s_nrej;
+        if (threadIdx.x == 0) {
+            *a.accept_len = len;
+            for (int j = len + 1; j < W1; ++j)
+                a.acc_nodes[j] = -1;
+        }
+        // the lowest retrieve row that starts with the accepted path
+        if (r < a.P) {
+            int same = 1;
+            for (int j = 0; j <= len; ++j)
+                same &= a.retrieve[r * W1 + j] == (j == 0 ? 0 : a.acc_nodes[j]);
+            s_len[r] = same;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int b = 0;
+            for (int q = 0; q < a.P; ++q)
+                if (s_len[q]) { b = q; break; }
+            *a.best = b;
+        }
+        // Gumbel-max over the tokens that were not struck out at the last node
+        const float inv_tau = (float)(1.0 / tau);
+        const float *lp = a.logits + (size_t)last_node * a.V;
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int v = threadIdx.x; v < a.V; v += blockDim.x) {
+            bool struck = false;
+            for (int q = 0; q < nrej; ++q)
+                struck |= s_rej[q] == v;
+            if (struck)
+                continue;
+            const float sc = __fadd_rn(__fmul_rn(lp[v], inv_tau), a.gumbel[v]);
+            if (better_f(sc, v, bv, bi)) { bv = sc; bi = v; }
+        }
+        const int am = block_argmax(bv, bi, sv, si);
+        if (threadIdx.x == 0)
+            *a.next_root = am;
+        return;
+    }
     if (r < a.P) {
         int len = 0;
         for (int j = 1; j < W; ++j) {
@@ -264,11 +359,12 @@ select_path_kernel(PosteriorArgs a, int typical, double tau, double eps, double 
 
 void launch_evaluate_posterior(const PosteriorArgs &a, cudaStream_t s)
 {
-    int typical = (a.mode == MEDUSA_TYPICAL && a.temperature > 0.f) ? 1 : 0;
+    const int rejection = (a.mode == MEDUSA_REJECTION && a.temperature > 0.f) ? 1 : 0;
+    int typical = ((a.mode == MEDUSA_TYPICAL && a.temperature > 0.f) || rejection) ? 1 : 0;
     double tau = typical ? (double)a.temperature : 1.0;
     launch_pdl(node_stats_kernel, dim3(a.T, typical ? a.stat_slices : 1), dim3(1024), 0, s, a.logits, a.V, typical, tau, a.node_argmax,
                reinterpret_cast<NodePart *>(a.node_part));
-    launch_pdl(select_path_kernel, dim3(1), dim3(256), 0, s, a, typical, tau, (double)a.eps, (double)a.delta);
+    launch_pdl(select_path_kernel, dim3(1), dim3(256), 0, s, a, typical, tau, (double)a.eps, (double)a.delta, rejection);
 }
 
 __global__ void __launch_bounds__(1024) argmax_row_kernel(const float *__restrict__ logits, int V, int row, int32_t *out)

@@ -203,6 +203,12 @@ def heads_inputs(d: int, V: int, K: int, seed: int, dtype: str = "bf16", std: fl
     )
 
 
+def uniform_noise(steps: int, n: int, seed: int) -> np.ndarray:
+    """Uniform numbers in [0, 1), float32 [steps][n] (one per tree node and step: the draws of rejection sampling)."""
+    u = rng(seed, "uniform").random((steps, n), dtype=np.float64).astype(np.float32)
+    return np.minimum(u, np.float32(0.99999994))
+
+
 def gumbel_noise(steps: int, V: int, seed: int) -> np.ndarray:
     """Standard Gumbel noise -log(-log u), float32 [steps][V], for replayable sampling."""
     u = rng(seed, "gumbel").random((steps, V), dtype=np.float64)

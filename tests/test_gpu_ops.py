@@ -281,6 +281,100 @@ def test_evaluate_posterior_bit_exact(oracle, tree_name):
     ctx.close()
 
 
+def _distinct_sibling_tokens(g, ot, logits, V, likely=0.7):
+    """Tree tokens as top-k picks give them: siblings distinct; with probability `likely` a child carries one of its
+    parent's most probable tokens, so that rejection sampling accepts paths of every length."""
+    T = ot["T"]
+    tok = np.zeros(T, dtype=np.int32)
+    tok[0] = int(g.integers(0, V))
+    for n in range(T):
+        kids = [c for c in range(T) if c != n and ot["parent"][c] == n]
+        if not kids:
+            continue
+        order = np.argsort(-logits[n], kind="stable")
+        pool = list(order[:len(kids)]) if g.random() < likely else list(g.permutation(V)[:len(kids)])
+        tok[kids] = np.array(pool, dtype=np.int32)
+    return tok
+
+
+@pytest.mark.parametrize("tree_name", ["dense22", "sparse64_d4", "sparse64_d5", "sparse256_d5"])
+def test_rejection_sampling_acceptance_bit_exact(oracle, tree_name):
+    """Rejection sampling over the tree (Sec. 1 / Sec. 2.3.1, first paragraph; deterministic drafts): accepted path,
+    row, and the token sampled from the residual equal the oracle's on identical logits, uniforms and Gumbel noise."""
+    torch, B, U = _gpu()
+    V = 1000
+    spec = I.LARGE_TREE_SPECS[tree_name] if tree_name in I.LARGE_TREE_SPECS else I.TREE_SPECS[tree_name]
+    cfg = dict(n_layers=0, d=64, n_heads=1, head_dim=64, ffn=8, vocab=V, n_medusa=5, max_tree_nodes=spec["n_nodes"])
+    ctx = U.make_ctx(cfg, "f32", 0, spec)
+    ot = oracle.build_tree_buffers(oracle.default_tree_paths(**spec))
+    T = ot["T"]
+    g = I.rng(71, tree_name)
+    f32 = lambda x: float(np.float32(x))
+    lens = []
+    n_masked = 0
+    for trial in range(16):
+        logits = (2.5 * g.standard_normal((T, V))).astype(np.float32)
+        tok = _distinct_sibling_tokens(g, ot, logits, V)
+        noise = I.gumbel_noise(1, V, 300 + trial)[0]
+        for tau in (0.7, 1.3, 0.05):
+            u = g.random(T).astype(np.float32)
+            if trial % 4 == 3:
+                u[:] = np.float32(0.99999994)  # everything rejected: the residual sample excludes the root's children
+            ref = oracle.evaluate_posterior(logits, tok, ot, mode=oracle.REJECTION, tau=f32(tau), gumbel=noise, uniform=u)
+            assert ref["min_margin"] > 1e-9, "a uniform within rounding of its acceptance probability: change the seed"
+            got = _posterior_gpu(torch, B, ctx, logits, tok, B.REJECTION, tau, 0.0, 0.0, np.concatenate([noise, u]))
+            for k in ("best", "accept_len", "next_root"):
+                assert got[k] == ref[k], (trial, tau, k, got, ref)
+            assert got["acc_nodes"].tolist() == ref["acc_nodes"].tolist()
+            lens.append(ref["accept_len"])
+            # did the mask matter?  (the unmasked sample would have been a rejected token)
+            last = ref["acc_nodes"][ref["accept_len"]]
+            plain = int(np.argmax((logits[last] * np.float32(1.0 / f32(tau))).astype(np.float32) + noise))
+            n_masked += plain != ref["next_root"]
+    assert max(lens) >= min(3, ot["depth"]) and min(lens) == 0, "the draws must exercise short and long accepted paths"
+    assert n_masked > 0, "the draws must exercise the exclusion of rejected tokens from the residual sample"
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_rejection_sampling_hand_vectors_and_refusals(oracle):
+    import json
+    import os
+    torch, B, U = _gpu()
+    fx = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "rejection_sampling_vectors.json")))["cases"]
+    for c in fx:
+        m = len(c["children_tokens"])
+        paths = np.array([[i] for i in range(m)], dtype=np.int32)
+        V = 8  # the fixture's four logits, padded with very unlikely tokens
+        cfg = dict(n_layers=0, d=64, n_heads=1, head_dim=64, ffn=8, vocab=V, n_medusa=1)
+        ctx = B.Context(cfg, B.F32, 0)
+        ctx.build_tree_buffers(paths)
+        row = np.full(V, -80.0, dtype=np.float32)
+        row[:4] = c["logits"]
+        logits = np.tile(row, (m + 1, 1))
+        tok = np.array([0] + c["children_tokens"], dtype=np.int32)
+        for tr in c["trials"]:
+            u = np.array([0.0] + tr["uniform"], dtype=np.float32)
+            got = _posterior_gpu(torch, B, ctx, logits, tok, B.REJECTION, c["tau"], 0.0, 0.0,
+                                 np.concatenate([np.zeros(V, np.float32), u]))
+            k = tr["accepted_child"]
+            assert got["accept_len"] == (1 if k >= 0 else 0)
+            assert got["acc_nodes"].tolist() == ([0, 1 + k] if k >= 0 else [0, -1])
+            if k < 0:  # zero noise: the most probable token that was not rejected
+                rest = [v for v in range(4) if v not in c["children_tokens"]]
+                assert got["next_root"] == max(rest, key=lambda v: c["logits"][v])
+        # refusals: no noise row, temperature zero
+        lg = torch.from_numpy(logits).cuda()
+        tk = torch.from_numpy(tok).cuda()
+        out = torch.zeros(8, dtype=torch.int32, device="cuda")
+        with pytest.raises(B.MedusaError):
+            ctx.evaluate_posterior(lg, tk, B.AcceptParams(mode=B.REJECTION, temperature=0.7), None, out[0:1], out[1:2], out[2:3], out[3:])
+        noise = torch.zeros(V + m + 1, device="cuda")
+        with pytest.raises(B.MedusaError):
+            ctx.evaluate_posterior(lg, tk, B.AcceptParams(mode=B.REJECTION, temperature=0.0), noise, out[0:1], out[1:2], out[2:3], out[3:])
+        ctx.close()
+
+
 def test_evaluate_posterior_planted_paths(oracle):
     torch, B, U = _gpu()
     V = 64
