@@ -1,7 +1,8 @@
 """ctypes front end of the CPU oracle (medusa_oracle.c).  TEST INFRASTRUCTURE, NOT THE PRODUCT.
 
 Only tests, the smoke check and the benchmark's CPU-baseline leg may import this module.  It holds
-no arithmetic of its own: every function marshals numpy arrays into the C oracle and back.
+no arithmetic of its own: every function marshals numpy arrays into the C oracle and back (the heads' training
+objective, re-exported at the end, is the one exception: it is written out in numpy in medusa1_training.py).
 """
 from __future__ import annotations
 
@@ -442,3 +443,7 @@ def rmsnorm(x, g, eps=1e-5):
     y = np.zeros_like(x)
     lib().ora_rmsnorm(_p(x), _p(g), C.c_int32(x.size), C.c_double(eps), _p(y))
     return y
+
+
+# the training objective of the heads (Sec. 2.2.1, Eq. 1) is written out in numpy in a module of its own
+from .medusa1_training import medusa1_loss_and_grads  # noqa: E402,F401

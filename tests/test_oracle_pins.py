@@ -921,3 +921,91 @@ def test_rejection_sampling_at_low_temperature_is_greedy(oracle):
         rj = oracle.evaluate_posterior(logits, tok, t, mode=oracle.REJECTION, tau=1e-3, gumbel=np.zeros(V, np.float32), uniform=u)
         assert rj["accept_len"] == gr["accept_len"] and rj["next_root"] == gr["next_root"]
         assert rj["acc_nodes"].tolist() == gr["acc_nodes"].tolist()
+
+
+# ----------------------------------------------------------------------------- Medusa-1 head training (Sec. 2.2.1, Eq. 1)
+
+def _train_case(seed, N=24, d=16, V=40, K=3):
+    g = I.rng(seed, "train")
+    h = g.standard_normal((N, d))
+    W1 = 0.3 * g.standard_normal((K, d, d))
+    W2 = 0.3 * g.standard_normal((K, V, d))
+    y = g.integers(0, V, size=(K, N))
+    for k in range(K):  # the last k + 1 positions of a sequence have no token that far ahead
+        y[k, N - (k + 1):] = -1
+    return h, W1, W2, y
+
+
+def test_medusa1_loss_matches_torch_cross_entropy_and_autograd(oracle):
+    torch = pytest.importorskip("torch")
+    h, W1, W2, y = _train_case(3)
+    K = W1.shape[0]
+    lam = [0.8 ** (k + 1) for k in range(K)]
+    r = oracle.medusa1_loss_and_grads(h, W1, W2, y)
+    th = torch.tensor(h, dtype=torch.float64)
+    t1 = torch.tensor(W1, dtype=torch.float64, requires_grad=True)
+    t2 = torch.tensor(W2, dtype=torch.float64, requires_grad=True)
+    total = 0.0
+    for k in range(K):
+        x = th + torch.nn.functional.silu(th @ t1[k].T)
+        lk = torch.nn.functional.cross_entropy(x @ t2[k].T, torch.tensor(y[k]), ignore_index=-1, reduction="mean")
+        assert abs(float(lk.detach()) - r["loss_per_head"][k]) < 1e-12
+        total = total + lam[k] * lk
+    total.backward()
+    assert abs(float(total.detach()) - r["loss"]) < 1e-12
+    assert np.abs(t1.grad.numpy() - r["grad_w1"]).max() < 1e-12
+    assert np.abs(t2.grad.numpy() - r["grad_w2"]).max() < 1e-12
+
+
+def test_medusa1_gradient_by_finite_differences(oracle):
+    h, W1, W2, y = _train_case(4, N=10, d=8, V=12, K=2)
+    r = oracle.medusa1_loss_and_grads(h, W1, W2, y)
+    g = I.rng(5, "fd")
+    eps = 1e-6
+    for which, W, grad in (("w1", W1, r["grad_w1"]), ("w2", W2, r["grad_w2"])):
+        for _ in range(12):
+            idx = tuple(int(g.integers(0, n)) for n in W.shape)
+            Wp, Wm = W.copy(), W.copy()
+            Wp[idx] += eps
+            Wm[idx] -= eps
+            a = (W1, Wp) if which == "w2" else (Wp, W2)
+            b = (W1, Wm) if which == "w2" else (Wm, W2)
+            fd = (oracle.medusa1_loss_and_grads(h, a[0], a[1], y)["loss"] - oracle.medusa1_loss_and_grads(h, b[0], b[1], y)["loss"]) / (2 * eps)
+            assert abs(fd - grad[idx]) < 1e-7, (which, idx, fd, grad[idx])
+
+
+def test_medusa1_closed_forms(oracle):
+    # zero weights: every head predicts the uniform distribution, loss_k = log V, and the gradient of W2_k is
+    # lambda_k * mean_n (1/V - onehot(y_n)) h_n^T; the gradient of W1 vanishes with W2
+    h, W1, W2, y = _train_case(6)
+    K, V, d = W2.shape
+    r = oracle.medusa1_loss_and_grads(h, np.zeros_like(W1), np.zeros_like(W2), y)
+    assert np.allclose(r["loss_per_head"], math.log(V), atol=1e-13)
+    assert abs(r["loss"] - sum(0.8 ** (k + 1) for k in range(K)) * math.log(V)) < 1e-12
+    assert np.abs(r["grad_w1"]).max() == 0.0
+    for k in range(K):
+        rows = np.nonzero(y[k] >= 0)[0]
+        ref = np.zeros((V, d))
+        for n in rows:
+            ref += (1.0 / V) * h[n][None, :]
+            ref[y[k][n]] -= h[n]
+        ref *= 0.8 ** (k + 1) / len(rows)
+        assert np.abs(r["grad_w2"][k] - ref).max() < 1e-13
+    # lambda scales a head's loss and gradient and nothing else; ignored positions change nothing
+    r1 = oracle.medusa1_loss_and_grads(h, W1, W2, y, lam=[1.0, 0.0, 0.5])
+    r2 = oracle.medusa1_loss_and_grads(h, W1, W2, y, lam=[2.0, 0.0, 0.5])
+    assert np.allclose(r2["grad_w1"][0], 2 * r1["grad_w1"][0]) and np.abs(r1["grad_w2"][1]).max() == 0.0
+    assert np.allclose(r2["grad_w2"][2], r1["grad_w2"][2])
+    h2 = h.copy()
+    h2[-1] += 5.0  # the last position carries no label for any head
+    r3 = oracle.medusa1_loss_and_grads(h2, W1, W2, y)
+    r0 = oracle.medusa1_loss_and_grads(h, W1, W2, y)
+    assert r3["loss"] == r0["loss"] and np.array_equal(r3["grad_w2"], r0["grad_w2"])
+    # a head whose logits already put all mass on the labels has (almost) no loss and no gradient
+    big = np.zeros_like(W2)
+    hh = np.eye(d)[:8]
+    yy = np.tile(np.arange(8), (K, 1))
+    for k in range(K):
+        big[k, np.arange(8), np.arange(8)] = 60.0
+    rz = oracle.medusa1_loss_and_grads(hh, np.zeros_like(W1), big, yy)
+    assert rz["loss"] < 1e-20 and np.abs(rz["grad_w2"]).max() < 1e-20
