@@ -347,6 +347,27 @@ int32_t medusa_generate(medusa_ctx *ctx, const int32_t *prompt_host, int32_t n_p
                         const medusa_accept_params *params, const float *gumbel_host, int32_t *out_tokens_host,
                         int32_t *emitted_per_step_host, int32_t *steps_host);
 
+/* ---- training of the heads with a frozen backbone (paper Sec. 2.2.1, Eq. 1) --------------------------- */
+
+/* Forward and backward pass of the Medusa-1 objective over N positions:
+ *   L = sum_k lambda_k * mean_n( -log p_n^(k)(labels[k][n]) ),  p^(k) = softmax(W2_k (h + SiLU(W1_k h)))  (Sec. 2.1.1),
+ * the mean taken over the positions whose label is >= 0 (the paper sums over the positions of a sequence; the mean is
+ * the reading taken so that the value does not depend on N), and its gradient with respect to W1_k and W2_k of the
+ * registered weights (the backbone is frozen: `hidden` is a constant).
+ * hidden: device [N][d] in the context's dtype, the backbone's last hidden states (the heads' input); labels: device
+ * int32 [K][N], labels[k][n] = the token head k + 1 should predict at position n (the token k + 2 positions after the
+ * one that produced hidden[n]), -1 where there is none; lambda_host: HOST float [K], NULL = 0.8^(k+1).
+ * Outputs (device, overwritten): loss float [K + 1] (per-head mean cross-entropy, then L); grad_w1 float [K][d][d];
+ * grad_w2 float [K][V][d] (same [out][in] layout as the weights).
+ * bf16 contexts with heads only, d a multiple of 256 and V a multiple of 128 (SHAPE otherwise).  Arithmetic: the five
+ * projections per head run on the tensor cores with bf16 operands and float accumulation -- the operand that takes the
+ * token position of the kernel is a split bf16 pair (h1, dz) or exact bf16 (h), the streamed operand one bf16 plane
+ * (weights as stored; dz^T, da^T and h1^T rounded) -- everything else in float; positions are processed 256 at a time
+ * and the gradients accumulated in position order.  Allocates its workspace (about 1 GB at the 7B shape) on the first
+ * call; enqueued on the context's stream, nothing is synchronised. */
+int32_t medusa_heads_loss_and_grads(medusa_ctx *ctx, const void *hidden, const int32_t *labels, int32_t N,
+                                    const float *lambda_host, float *loss, float *grad_w1, float *grad_w2);
+
 #ifdef __cplusplus
 }
 #endif

@@ -8,6 +8,7 @@ from __future__ import annotations
 
 import numpy as np
 
+
 def medusa1_loss_and_grads(h, W1, W2, labels, lam=None):
     """The Medusa-1 objective (Sec. 2.2.1, Eq. 1: frozen backbone, cross-entropy of every head against the token
     k + 1 positions ahead, weighted by lambda_k) and its gradient with respect to the heads' weights, in float64.
@@ -15,8 +16,8 @@ def medusa1_loss_and_grads(h, W1, W2, labels, lam=None):
     h [N][d]: the backbone's last hidden states at N positions (constants: the backbone is frozen).
     W1 [K][d][d], W2 [K][V][d]: the heads of Sec. 2.1.1, p^(k) = softmax(W2_k (h + SiLU(W1_k h))).
     labels [K][N] int: labels[k][n] = the token head k + 1 should predict at position n, or -1 where the sequence has
-    no such token (ignored).  lam [K]: lambda_k; default 0.8^k for k = 1..K (the paper's "k-th power of a constant
-    like 0.8").  Where the paper sums over the positions of one sequence, the reading here is the mean over the
+    no such token (ignored).  lam [K]: lambda_k; default 0.8^k for k = 1..K (Sec. 2.2.1 weights the heads by
+    powers of a constant and names 0.8).  Where the paper sums over the positions of one sequence, the reading here is the mean over the
     labelled positions of each head, so that the value does not depend on the batch size:
         L = sum_k lambda_k * mean_n( -log p_n^(k)(labels[k][n]) ).
     -> dict(loss_per_head [K], loss, grad_w1 [K][d][d], grad_w2 [K][V][d])

@@ -234,6 +234,13 @@ class Context:
         self._check(lib().medusa_decode_step_batch(self.handle, C.byref(params), _ptr(gumbel), C.c_int32(int(max_commit)),
                                                    _ptr(emitted_host), _ptr(n_emitted_host)))
 
+    def heads_loss_and_grads(self, hidden, labels, loss, grad_w1, grad_w2, lam=None):
+        """Medusa-1 objective and its gradient w.r.t. the heads (device tensors; lam: host floats [K] or None)."""
+        n = int(hidden.shape[0])
+        la = None if lam is None else np.ascontiguousarray(lam, dtype=np.float32)
+        self._check(lib().medusa_heads_loss_and_grads(self.handle, _ptr(hidden), _ptr(labels), C.c_int32(n), _ptr(la),
+                                                      _ptr(loss), _ptr(grad_w1), _ptr(grad_w2)))
+
     def generate(self, prompt_host: np.ndarray, G: int, params: AcceptParams, gumbel_host=None) -> dict:
         prompt = np.ascontiguousarray(prompt_host, dtype=np.int32)
         out = np.zeros(max(G, 1), dtype=np.int32)

@@ -16,7 +16,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libmedusa_b200.so")
-SOURCES = ["api.cu", "gemm_tc.cu", "simt_kernels.cu", "attention.cu", "attention_flash.cu", "attention_tc.cu", "heads.cu", "posterior.cu", "tree_host.cpp"]
+SOURCES = ["api.cu", "gemm_tc.cu", "simt_kernels.cu", "attention.cu", "attention_flash.cu", "attention_tc.cu", "heads.cu", "posterior.cu", "train_heads.cu", "tree_host.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -110,7 +110,7 @@ struct medusa_ctx {
 
     // Whole-step CUDA graphs (medusa_decode_step).  Everything a step launches depends on the host only through
     // the values in StepKey (the cache length is read on the device); the second consecutive step with the same key is captured from the stream into an
-    // executable graph, and later steps with that key replay it.  MEDUSA_STEP_GRAPH=0 turns this off.
+    // executable graph, and later steps with that key replay it.  MEDUSA_OPT_STEP_GRAPHS = 0 turns this off.
     struct StepKey {
         int32_t max_commit, has_gumbel, seq;
         medusa_accept_params p;
@@ -122,6 +122,24 @@ struct medusa_ctx {
         int64_t launches[MEDUSA_PROF_CATEGORIES];  // what one replay adds to the launch accounting
         uint64_t used;
     };
+    // Workspace of the heads' training pass (medusa_heads_loss_and_grads), allocated on its first call: 256 positions
+    // per chunk.  "planes" buffers are split activations [2][rows][width] (hi plane, lo plane).
+    struct TrainWs {
+        bool ready = false;
+        void *Hp = nullptr, *HT = nullptr;      // hidden states [2][256][d] (hi used) and their transpose [2][d][256]
+        void *H1p = nullptr, *H1T = nullptr;    // h1 = h + SiLU(W1 h) [2][256][d]; transpose of its hi plane [2][d][256]
+        float *A = nullptr, *part = nullptr;    // W1 h [256][d]; partial planes of the two stream-K projections
+        float *Z = nullptr;                     // logits [256][V]
+        void *dZp = nullptr, *dZT = nullptr;    // gradient of the logits [2][256][V]; transpose of its hi plane [V][256]
+        void *W2T = nullptr;                    // W2_k transposed [d][V]
+        void *dA = nullptr, *dAT = nullptr;     // gradient of W1 h [256][d] and transposed [d][256]
+        float *row_loss = nullptr;
+        int32_t *n_valid = nullptr;
+        size_t part_planes = 0;
+        TensorMap mHp, mHT, mH1p, mH1T, mdZp, mdZT, mW2T, mdAT;
+        std::vector<TensorMap> mW1, mW2;        // per head
+        const void *w1_of = nullptr, *w2_of = nullptr;  // the weight pointers those per-head maps were encoded for
+    } train;
     std::vector<StepGraph> step_graphs;
     StepKey last_key{};
     bool have_last_key = false;
@@ -1283,6 +1301,139 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
     }
     point_at(c, keep);
     return rc;
+}
+
+// ============================================================================ training of the heads (Sec. 2.2.1, Eq. 1)
+
+static constexpr int TRAIN_ROWS = 256;  // positions per chunk: four token tiles, one weight stream with a single plane
+
+// One projection over T token rows of a split activation (its map covers [2 * x_rows][K]) against a streamed operand of
+// Nw rows: launches of up to 256 rows (one plane) or 128 rows (two planes), all with the same plan; every launch is
+// fully serialised behind the kernel before it, because the streamed operand may have been written by that kernel.
+static int32_t train_gemm(medusa_ctx *c, const TensorMap *mapX, int x_rows, const TensorMap *mapW, int Nw, int K, float *P,
+                          size_t plane_stride, int ldy, int T, bool whole_tiles, int planes, PlaneDesc *pd, int out_t = 0)
+{
+    const int RT = gemm_tc_row_tiles(T, planes), rows_per_launch = RT * TREE_ROWS;
+    *pd = gemm_tc_plan(1, Nw, K, whole_tiles, (long long)plane_stride, 0, RT, planes);
+    if (!whole_tiles && (size_t)pd->n_max > c->train.part_planes)
+        return fail(c, MEDUSA_ERR_SHAPE, "training projection needs %d partial planes, the workspace holds %zu", pd->n_max, c->train.part_planes);
+    const TensorMap *maps[3] = {mapW, mapW, mapW};
+    for (int r0 = 0; r0 < T; r0 += rows_per_launch) {
+        const int Tt = T - r0 < rows_per_launch ? T - r0 : rows_per_launch;
+        cudaError_t e = cudaSuccess;
+        // out_t: the result goes transposed to P[n * ldy + token] (stored, or accumulated with out_t == 2)
+        PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, 1, Nw, K, *pd, out_t ? P + r0 : P + (size_t)r0 * ldy, ldy, Tt, 0,
+                                               c->d_state + ST_STATUS, c->stream, 0, c->spin_limit, 0, r0, x_rows + r0, RT, planes, true,
+                                               out_t, ldy));
+        if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "training projection launch failed: %s", cudaGetErrorString(e));
+    }
+    return MEDUSA_OK;
+}
+
+static int32_t train_weight_maps(medusa_ctx *c)
+{
+    medusa_ctx::TrainWs &w = c->train;
+    if (w.w1_of == c->w.medusa_w1 && w.w2_of == c->w.medusa_w2) return MEDUSA_OK;
+    const size_t d = c->m.d, V = c->m.vocab, K = c->m.n_medusa;
+    w.mW1.resize(K);
+    w.mW2.resize(K);
+    for (size_t k = 0; k < K; ++k)
+        if (!make_weight_map(&w.mW1[k], (const char *)c->w.medusa_w1 + k * d * d * 2, (int)d, (int)d) ||
+            !make_weight_map(&w.mW2[k], (const char *)c->w.medusa_w2 + k * V * d * 2, (int)V, (int)d))
+            return fail(c, MEDUSA_ERR_CUDA, "training workspace: tensor map encoding failed");
+    w.w1_of = c->w.medusa_w1;
+    w.w2_of = c->w.medusa_w2;
+    return MEDUSA_OK;
+}
+
+static int32_t train_workspace(medusa_ctx *c)
+{
+    medusa_ctx::TrainWs &w = c->train;
+    TRY(train_weight_maps(c));  // the heads' weights may have been registered anew since the last call
+    if (w.ready) return MEDUSA_OK;
+    const medusa_model_desc &m = c->m;
+    const size_t d = m.d, V = m.vocab, R = TRAIN_ROWS, K = m.n_medusa;
+    TRY(dev_alloc_bytes(c, &w.Hp, 2 * R * d * 2));
+    TRY(dev_alloc_bytes(c, &w.HT, 2 * d * R * 2));
+    TRY(dev_alloc_bytes(c, &w.H1p, 2 * R * d * 2));
+    TRY(dev_alloc_bytes(c, &w.H1T, 2 * d * R * 2));
+    TRY(dev_alloc(c, &w.A, R * d));
+    TRY(dev_alloc(c, &w.Z, R * V));
+    TRY(dev_alloc_bytes(c, &w.dZp, 2 * R * V * 2));
+    TRY(dev_alloc_bytes(c, &w.dZT, V * R * 2));
+    TRY(dev_alloc_bytes(c, &w.W2T, d * V * 2));
+    TRY(dev_alloc_bytes(c, &w.dA, R * d * 2));
+    TRY(dev_alloc_bytes(c, &w.dAT, d * R * 2));
+    TRY(dev_alloc(c, &w.row_loss, R));
+    TRY(dev_alloc(c, &w.n_valid, K));
+    // the two projections whose output has only d columns (32 tiles at d = 4096) are cut stream-K over all CTAs
+    const PlaneDesc p1 = gemm_tc_plan(1, (int)d, (int)d, false, (long long)(R * d), 0, 4, 1);
+    const PlaneDesc p4 = gemm_tc_plan(1, (int)d, (int)V, false, (long long)(R * d), 0, 2, 2);
+    w.part_planes = (size_t)(p1.n_max > p4.n_max ? p1.n_max : p4.n_max);
+    TRY(dev_alloc(c, &w.part, w.part_planes * R * d));
+    bool ok = make_act_map(&w.mHp, w.Hp, (int)d, (int)R) && make_act_map(&w.mHT, w.HT, (int)R, (int)d) &&
+              make_act_map(&w.mH1p, w.H1p, (int)d, (int)R) && make_act_map(&w.mH1T, w.H1T, (int)R, (int)d) &&
+              make_act_map(&w.mdZp, w.dZp, (int)V, (int)R) && make_weight_map(&w.mdZT, w.dZT, (int)V, (int)R) &&
+              make_weight_map(&w.mW2T, w.W2T, (int)d, (int)V) && make_weight_map(&w.mdAT, w.dAT, (int)d, (int)R);
+    if (!ok) return fail(c, MEDUSA_ERR_CUDA, "training workspace: tensor map encoding failed");
+    w.ready = true;
+    return MEDUSA_OK;
+}
+
+extern "C" int32_t medusa_heads_loss_and_grads(medusa_ctx *c, const void *hidden, const int32_t *labels, int32_t N,
+                                               const float *lambda_host, float *loss, float *grad_w1, float *grad_w2)
+{
+    TRY(check_ready(c, false, true));
+    if (!hidden || !labels || !loss || !grad_w1 || !grad_w2 || N < 1)
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_heads_loss_and_grads: null pointer or no positions");
+    const medusa_model_desc &m = c->m;
+    const int d = m.d, V = m.vocab, K = m.n_medusa, R = TRAIN_ROWS;
+    if (!c->use_tc || K < 1 || d % R != 0 || V % 128 != 0 || !c->w.medusa_w1 || !c->w.medusa_w2)
+        return fail(c, MEDUSA_ERR_SHAPE, "medusa_heads_loss_and_grads: needs a bf16 context with heads, d a multiple of 256 and V a multiple of 128");
+    if (!aligned16(hidden) || !aligned16(grad_w1) || !aligned16(grad_w2))
+        return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_heads_loss_and_grads: tensors must be 16-byte aligned");
+    MEDUSA_CUDA(c, cudaSetDevice(c->device));
+    TRY(train_workspace(c));
+    medusa_ctx::TrainWs &w = c->train;
+    cudaStream_t s = c->stream;
+    const size_t dd = (size_t)d * d, Vd = (size_t)V * d, Rd = (size_t)R * d, RV = (size_t)R * V;
+    MEDUSA_CUDA(c, cudaMemsetAsync(loss, 0, (size_t)(K + 1) * sizeof(float), s));
+    PROF(c, PC_ELEMWISE, 1, launch_count_valid(labels, K, N, w.n_valid, s));
+    for (int k = 0; k < K; ++k) {
+        const float lambda = lambda_host ? lambda_host[k] : (float)pow(0.8, (double)(k + 1));
+        // W2_k^T, the streamed operand of dh1 = dz W2_k
+        PROF(c, PC_ELEMWISE, 1, launch_transpose_bf16((const char *)c->w.medusa_w2 + (size_t)k * Vd * 2, V, d, d, w.W2T, V, s));
+        for (int n0 = 0; n0 < N; n0 += R) {
+            const int rows = N - n0 < R ? N - n0 : R;
+            // this chunk's hidden states (rows beyond the chunk are zero: they contribute nothing to any sum over positions)
+            MEDUSA_CUDA(c, cudaMemcpyAsync(w.Hp, (const char *)hidden + (size_t)n0 * d * 2, (size_t)rows * d * 2, cudaMemcpyDeviceToDevice, s));
+            if (rows < R)
+                MEDUSA_CUDA(c, cudaMemsetAsync((char *)w.Hp + (size_t)rows * d * 2, 0, (size_t)(R - rows) * d * 2, s));
+            PROF(c, PC_ELEMWISE, 1, launch_transpose_bf16(w.Hp, R, d, d, w.HT, R, s));
+            PlaneDesc pd{};
+            // a = W1_k h   (h is exactly bf16: one plane)
+            TRY(train_gemm(c, &w.mHp, R, &w.mW1[k], d, d, w.part, Rd, d, R, false, 1, &pd));
+            PROF(c, PC_ELEMWISE, 1, launch_head_hidden_fwd(w.part, pd, w.Hp, w.A, w.H1p, (char *)w.H1p + Rd * 2, R, d, s));
+            PROF(c, PC_ELEMWISE, 1, launch_transpose_bf16(w.H1p, R, d, d, w.H1T, R, s));
+            // z = W2_k h1   (every CTA owns whole tiles: one plane, written straight into the logits buffer)
+            TRY(train_gemm(c, &w.mH1p, R, &w.mW2[k], V, d, w.Z, 0, V, R, true, 2, &pd));
+            PROF(c, PC_ELEMWISE, 1, launch_ce_grad(w.Z, V, labels + (size_t)k * N + n0, R, rows, w.n_valid + k, lambda, w.row_loss, w.dZp,
+                                                   (char *)w.dZp + RV * 2, s));
+            PROF(c, PC_ELEMWISE, 1, launch_loss_accumulate(w.row_loss, R, w.n_valid + k, lambda, loss + k, loss + K, s));
+            PROF(c, PC_ELEMWISE, 1, launch_transpose_bf16(w.dZp, R, V, V, w.dZT, R, s));
+            // gW2_k^T [d][V] = h1^T (d token rows) x dz^T (V streamed rows, K = the chunk's positions)
+            // (stored transposed by the projection's epilogue: straight into, or onto, gW2_k [V][d])
+            TRY(train_gemm(c, &w.mH1T, d, &w.mdZT, V, R, grad_w2 + (size_t)k * Vd, 0, d, d, true, 1, &pd, n0 > 0 ? 2 : 1));
+            // dh1 = dz W2_k
+            TRY(train_gemm(c, &w.mdZp, R, &w.mW2T, d, V, w.part, Rd, d, R, false, 2, &pd));
+            PROF(c, PC_ELEMWISE, 1, launch_head_hidden_bwd(w.part, pd, w.A, w.dA, R, d, s));
+            PROF(c, PC_ELEMWISE, 1, launch_transpose_bf16(w.dA, R, d, d, w.dAT, R, s));
+            // gW1_k^T [d][d] = h^T (d token rows) x da^T (d streamed rows)
+            TRY(train_gemm(c, &w.mHT, d, &w.mdAT, d, R, grad_w1 + (size_t)k * dd, 0, d, d, true, 1, &pd, n0 > 0 ? 2 : 1));
+        }
+    }
+    MEDUSA_LAUNCH_CHECK(c);
+    return MEDUSA_OK;
 }
 
 extern "C" int32_t medusa_generate(medusa_ctx *c, const int32_t *prompt_host, int32_t n_prompt, int32_t G,

@@ -199,7 +199,8 @@ struct SegmentIter {
 // tile of a stage feeds RT MMAs of N = 64 PL, one per token tile, into RT accumulators of 64 PL columns; the accumulators
 // are double-buffered, so a CTA holds 2 RT 64 PL tensor-memory columns: up to 256 leaves room for two CTAs per SM,
 // 512 (RT PL = 4) means one CTA per SM with a deeper ring.
-template <int RT, int PL>
+// OT: the result may be stored or accumulated transposed (a.out_t; the gradient projections of the heads' training)
+template <int RT, int PL, bool OT = false>
 __global__ void __launch_bounds__(THREADS, RT * PL <= 2 ? 2 : 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW0,
                const __grid_constant__ CUtensorMap mapW1, const __grid_constant__ CUtensorMap mapW2, GemmTcArgs a)
@@ -399,7 +400,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                         for (int i = 0; i < 32; ++i)
                             w[i] = 0u;  // +0.0f
                     }
-                    if (n_ok) {
+                    if (OT && n_ok && a.out_t) {
+                        // transposed result: this thread's 32 tokens are consecutive floats of row (col0 + n)
+                        float *o = a.P + (size_t)(col0 + n) * a.ldt + (tb + half * 32);
+                        if (all_rows) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                float4 r = a.out_t == 2 ? *reinterpret_cast<const float4 *>(o + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                r.x += __uint_as_float(v[i]) + __uint_as_float(w[i]);
+                                r.y += __uint_as_float(v[i + 1]) + __uint_as_float(w[i + 1]);
+                                r.z += __uint_as_float(v[i + 2]) + __uint_as_float(w[i + 2]);
+                                r.w += __uint_as_float(v[i + 3]) + __uint_as_float(w[i + 3]);
+                                *reinterpret_cast<float4 *>(o + i) = r;
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                const int t = tb + half * 32 + i;
+                                if (t >= a.row0 && t < a.T)
+                                    o[i] = (a.out_t == 2 ? o[i] : 0.f) + (__uint_as_float(v[i]) + __uint_as_float(w[i]));
+                            }
+                        }
+                    } else if (n_ok) {
                         float *o = out + (size_t)(tb + half * 32) * a.ldy;  // a warp writes 32 consecutive floats per token row
                         if (all_rows) {
 #pragma unroll
@@ -550,12 +572,20 @@ static GemmKernel gemm_kernel(int rt, int pl)
     if (pl == 2) return rt == 1 ? gemm_tc_kernel<1, 2> : gemm_tc_kernel<2, 2>;
     return rt == 1 ? gemm_tc_kernel<1, 1> : (rt == 2 ? gemm_tc_kernel<2, 1> : gemm_tc_kernel<4, 1>);
 }
+// the instantiation whose epilogue can store transposed: four token tiles, one plane
+static GemmKernel gemm_kernel_transposing()
+{
+    return gemm_tc_kernel<4, 1, true>;
+}
 
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
                            int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo, int row_tiles,
-                           int planes)
+                           int planes, bool serialize, int out_t, long long ldt)
 {
+    if (out_t && (pd.G != 0 || row_tiles < 4 || planes != 1))
+        return cudaErrorInvalidValue;  // a transposed result needs whole tiles (one plane, every element written once);
+                                       // only the four-tile single-plane kernel is built with that epilogue
     if (seg0_cols <= 0) seg0_cols = seg_cols;
     const int rt = row_tiles >= 4 && planes == 1 ? 4 : (row_tiles >= 2 ? 2 : 1), pl = planes == 1 ? 1 : 2;
     const int stages = cfg_stages(rt, pl);
@@ -568,6 +598,10 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
             if (e != cudaSuccess)
                 return e;
         }
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel_transposing(), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem_bytes(cfg_stages(4, 1), 4, 1));
+        if (e != cudaSuccess)
+            return e;
     }
     GemmTcArgs a;
     a.P = P;
@@ -589,6 +623,8 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     a.withhold = withhold;
     a.x_row_hi = x_row_hi;
     a.x_row_lo = x_row_lo;
+    a.out_t = out_t;
+    a.ldt = ldt;
     const CUtensorMap *w0 = (const CUtensorMap *)mapW[0];
     const CUtensorMap *w1 = (const CUtensorMap *)mapW[n_seg > 1 ? 1 : 0];
     const CUtensorMap *w2 = (const CUtensorMap *)mapW[n_seg > 2 ? 2 : 0];
@@ -599,10 +635,10 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = tuning_env("MEDUSA_NO_PDL") ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed = serialize || tuning_env("MEDUSA_NO_PDL") ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_kernel(rt, pl), *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
+    return cudaLaunchKernelEx(&cfg, out_t ? gemm_kernel_transposing() : gemm_kernel(rt, pl), *(const CUtensorMap *)mapX, *w0, *w1, *w2, a);
 }
 
 }  // namespace medusa

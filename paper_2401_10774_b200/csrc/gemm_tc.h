@@ -54,6 +54,8 @@ struct GemmTcArgs {
     uint32_t spin_limit;     // polls before a bounded wait gives up
     int withhold;            // test hook: CTA 0's producer issues no load at all, so its consumers' waits expire
     int x_row_hi, x_row_lo;  // rows of the activation tensor where this launch's 64 token rows start in the hi / lo plane
+    int out_t;               // 0: P[t][n];  1: P[n * ldt + t] = result (transposed store);  2: P[n * ldt + t] += result
+    long long ldt;           // row stride of the transposed output (whole-tile launches only)
 };
 
 // W: [N][K] bf16 row-major
@@ -78,6 +80,12 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
                            int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0, int x_row_hi = 0, int x_row_lo = 64,
-                           int row_tiles = 1, int planes = 2);
+                           int row_tiles = 1, int planes = 2, bool serialize = false, int out_t = 0, long long ldt = 0);
+// serialize: launch without programmatic dependent launch.  The kernel requests its streamed ("weight") operand BEFORE it
+// waits for the preceding kernel, which is right for constant weights; a launch whose streamed operand was written by
+// the preceding kernel (the gradient projections of the heads' training) must be fully serialised behind it.
+// out_t = 1 / 2 (plans with whole tiles only): the result is stored / accumulated transposed, P[n * ldt + t] with n the
+// streamed operand's row and t the token row counted from the launch's first one (P points at that column); every thread
+// of the epilogue then owns 32 consecutive floats of a row.
 
 }  // namespace medusa

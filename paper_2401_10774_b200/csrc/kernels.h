@@ -138,4 +138,17 @@ void launch_iota(int32_t *p, int n, cudaStream_t s);
 // out[0] = argmax of logits[row] (ties: lower index)
 void launch_argmax_row(const float *logits, int V, int row, int32_t *out, cudaStream_t s);
 
+
+// ---- training of the heads (paper Sec. 2.2.1, Eq. 1): the kernels around the projections, train_heads.cu
+void launch_head_hidden_fwd(const float *A_planes, const PlaneDesc &pd, const void *H, float *A, void *h1_hi, void *h1_lo, int rows,
+                            int d, cudaStream_t s);
+void launch_head_hidden_bwd(const float *dH1_planes, const PlaneDesc &pd, const float *A, void *dA, int rows, int d, cudaStream_t s);
+void launch_ce_grad(const float *Z, int V, const int32_t *labels, int rows, int rows_valid, const int32_t *n_valid, float lambda,
+                    float *row_loss, void *dz_hi, void *dz_lo, cudaStream_t s);
+void launch_loss_accumulate(const float *row_loss, int rows, const int32_t *n_valid, float lambda, float *loss_k, float *loss_total,
+                            cudaStream_t s);
+void launch_count_valid(const int32_t *labels, int K, int N, int32_t *n_valid, cudaStream_t s);
+// out[c][r] = in[r][c] for a row-major [R][C] bf16 matrix
+void launch_transpose_bf16(const void *in, int R, int Cc, long long ld_in, void *out, long long ld_out, cudaStream_t s);
+
 }  // namespace medusa
