@@ -362,9 +362,9 @@ int32_t medusa_generate(medusa_ctx *ctx, const int32_t *prompt_host, int32_t n_p
  * bf16 contexts with heads only, d a multiple of 256 and V a multiple of 128 (SHAPE otherwise).  Arithmetic: the five
  * projections per head run on the tensor cores with bf16 operands and float accumulation -- the operand that takes the
  * token position of the kernel is a split bf16 pair (h1, dz) or exact bf16 (h), the streamed operand one bf16 plane
- * (weights as stored; dz^T, da^T and h1^T rounded) -- everything else in float; positions are processed 256 at a time
- * and the gradients accumulated in position order.  Allocates its workspace (about 1 GB at the 7B shape) on the first
- * call; enqueued on the context's stream, nothing is synchronised. */
+ * (weights as stored; dz^T, da^T and h1^T rounded) -- everything else in float; positions are processed in chunks of up
+ * to 1024 and the gradients accumulated chunk by chunk in position order.  Allocates its workspace (about 0.8 GB at the
+ * 7B shape) on the first call; enqueued on the context's stream, nothing is synchronised. */
 int32_t medusa_heads_loss_and_grads(medusa_ctx *ctx, const void *hidden, const int32_t *labels, int32_t N,
                                     const float *lambda_host, float *loss, float *grad_w1, float *grad_w2);
 

@@ -122,23 +122,24 @@ struct medusa_ctx {
         int64_t launches[MEDUSA_PROF_CATEGORIES];  // what one replay adds to the launch accounting
         uint64_t used;
     };
-    // Workspace of the heads' training pass (medusa_heads_loss_and_grads), allocated on its first call: 256 positions
-    // per chunk.  "planes" buffers are split activations [2][rows][width] (hi plane, lo plane).
+    // Workspace of the heads' training pass (medusa_heads_loss_and_grads), allocated on its first call for chunks of up
+    // to 1024 positions (R below is the chunk size of the call).  "planes" buffers are split activations [2][rows][width] (hi plane, lo plane).
     struct TrainWs {
         bool ready = false;
-        void *Hp = nullptr, *HT = nullptr;      // hidden states [2][256][d] (hi used) and their transpose [2][d][256]
-        void *H1p = nullptr, *H1T = nullptr;    // h1 = h + SiLU(W1 h) [2][256][d]; transpose of its hi plane [2][d][256]
-        float *A = nullptr, *part = nullptr;    // W1 h [256][d]; partial planes of the two stream-K projections
-        float *Z = nullptr;                     // logits [256][V]
-        void *dZp = nullptr, *dZT = nullptr;    // gradient of the logits [2][256][V]; transpose of its hi plane [V][256]
+        void *Hp = nullptr, *HT = nullptr;      // hidden states [2][R][d] (hi used) and their transpose [2][d][R]
+        void *H1p = nullptr, *H1T = nullptr;    // h1 = h + SiLU(W1 h) [2][R][d]; transpose of its hi plane [2][d][R]
+        float *A = nullptr, *part = nullptr;    // W1 h [R][d]; partial planes of the two stream-K projections
+        float *Z = nullptr;                     // logits [R][V]
+        void *dZp = nullptr, *dZT = nullptr;    // gradient of the logits [2][R][V]; transpose of its hi plane [V][R]
         void *W2T = nullptr;                    // W2_k transposed [d][V]
-        void *dA = nullptr, *dAT = nullptr;     // gradient of W1 h [256][d] and transposed [d][256]
+        void *dA = nullptr, *dAT = nullptr;     // gradient of W1 h [R][d] and transposed [d][R]
         float *row_loss = nullptr;
         int32_t *n_valid = nullptr;
         size_t part_planes = 0;
         TensorMap mHp, mHT, mH1p, mH1T, mdZp, mdZT, mW2T, mdAT;
         std::vector<TensorMap> mW1, mW2;        // per head
         const void *w1_of = nullptr, *w2_of = nullptr;  // the weight pointers those per-head maps were encoded for
+        int R = 0;                              // chunk size the chunk buffers' maps were encoded for
     } train;
     std::vector<StepGraph> step_graphs;
     StepKey last_key{};
@@ -1305,7 +1306,10 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
 
 // ============================================================================ training of the heads (Sec. 2.2.1, Eq. 1)
 
-static constexpr int TRAIN_ROWS = 256;  // positions per chunk: four token tiles, one weight stream with a single plane
+// Positions per chunk: the contraction length of the two gradient projections, whose results (V x d and d x d floats)
+// are written once per chunk -- 1024 positions make them compute-bound instead of store-bound; a shorter batch takes
+// the next multiple of 256 (four token tiles, one weight stream with a single plane).
+static constexpr int TRAIN_ROWS_MAX = 1024;
 
 // One projection over T token rows of a split activation (its map covers [2 * x_rows][K]) against a streamed operand of
 // Nw rows: launches of up to 256 rows (one plane) or 128 rows (two planes), all with the same plan; every launch is
@@ -1346,13 +1350,27 @@ static int32_t train_weight_maps(medusa_ctx *c)
     return MEDUSA_OK;
 }
 
+// maps of the chunk buffers for chunks of R positions (R is the K extent of the transposed buffers)
+static int32_t train_chunk_maps(medusa_ctx *c, int R)
+{
+    medusa_ctx::TrainWs &w = c->train;
+    if (w.R == R) return MEDUSA_OK;
+    const int d = c->m.d, V = c->m.vocab;
+    const bool ok = make_act_map(&w.mHp, w.Hp, d, R) && make_act_map(&w.mHT, w.HT, R, d) && make_act_map(&w.mH1p, w.H1p, d, R) &&
+                    make_act_map(&w.mH1T, w.H1T, R, d) && make_act_map(&w.mdZp, w.dZp, V, R) && make_weight_map(&w.mdZT, w.dZT, V, R) &&
+                    make_weight_map(&w.mW2T, w.W2T, d, V) && make_weight_map(&w.mdAT, w.dAT, d, R);
+    if (!ok) return fail(c, MEDUSA_ERR_CUDA, "training workspace: tensor map encoding failed");
+    w.R = R;
+    return MEDUSA_OK;
+}
+
 static int32_t train_workspace(medusa_ctx *c)
 {
     medusa_ctx::TrainWs &w = c->train;
     TRY(train_weight_maps(c));  // the heads' weights may have been registered anew since the last call
     if (w.ready) return MEDUSA_OK;
     const medusa_model_desc &m = c->m;
-    const size_t d = m.d, V = m.vocab, R = TRAIN_ROWS, K = m.n_medusa;
+    const size_t d = m.d, V = m.vocab, R = TRAIN_ROWS_MAX, K = m.n_medusa;
     TRY(dev_alloc_bytes(c, &w.Hp, 2 * R * d * 2));
     TRY(dev_alloc_bytes(c, &w.HT, 2 * d * R * 2));
     TRY(dev_alloc_bytes(c, &w.H1p, 2 * R * d * 2));
@@ -1371,11 +1389,6 @@ static int32_t train_workspace(medusa_ctx *c)
     const PlaneDesc p4 = gemm_tc_plan(1, (int)d, (int)V, false, (long long)(R * d), 0, 2, 2);
     w.part_planes = (size_t)(p1.n_max > p4.n_max ? p1.n_max : p4.n_max);
     TRY(dev_alloc(c, &w.part, w.part_planes * R * d));
-    bool ok = make_act_map(&w.mHp, w.Hp, (int)d, (int)R) && make_act_map(&w.mHT, w.HT, (int)R, (int)d) &&
-              make_act_map(&w.mH1p, w.H1p, (int)d, (int)R) && make_act_map(&w.mH1T, w.H1T, (int)R, (int)d) &&
-              make_act_map(&w.mdZp, w.dZp, (int)V, (int)R) && make_weight_map(&w.mdZT, w.dZT, (int)V, (int)R) &&
-              make_weight_map(&w.mW2T, w.W2T, (int)d, (int)V) && make_weight_map(&w.mdAT, w.dAT, (int)d, (int)R);
-    if (!ok) return fail(c, MEDUSA_ERR_CUDA, "training workspace: tensor map encoding failed");
     w.ready = true;
     return MEDUSA_OK;
 }
@@ -1387,13 +1400,15 @@ extern "C" int32_t medusa_heads_loss_and_grads(medusa_ctx *c, const void *hidden
     if (!hidden || !labels || !loss || !grad_w1 || !grad_w2 || N < 1)
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_heads_loss_and_grads: null pointer or no positions");
     const medusa_model_desc &m = c->m;
-    const int d = m.d, V = m.vocab, K = m.n_medusa, R = TRAIN_ROWS;
-    if (!c->use_tc || K < 1 || d % R != 0 || V % 128 != 0 || !c->w.medusa_w1 || !c->w.medusa_w2)
+    const int d = m.d, V = m.vocab, K = m.n_medusa;
+    const int R = N >= TRAIN_ROWS_MAX ? TRAIN_ROWS_MAX : ((N + 255) / 256) * 256;  // positions per chunk
+    if (!c->use_tc || K < 1 || d % 256 != 0 || V % 128 != 0 || !c->w.medusa_w1 || !c->w.medusa_w2)
         return fail(c, MEDUSA_ERR_SHAPE, "medusa_heads_loss_and_grads: needs a bf16 context with heads, d a multiple of 256 and V a multiple of 128");
     if (!aligned16(hidden) || !aligned16(grad_w1) || !aligned16(grad_w2))
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_heads_loss_and_grads: tensors must be 16-byte aligned");
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
     TRY(train_workspace(c));
+    TRY(train_chunk_maps(c, R));
     medusa_ctx::TrainWs &w = c->train;
     cudaStream_t s = c->stream;
     const size_t dd = (size_t)d * d, Vd = (size_t)V * d, Rd = (size_t)R * d, RV = (size_t)R * V;

@@ -5,7 +5,12 @@
 //
 // Shape of the computation ("swap AB"): the weight rows are the MMA's M dimension, the tokens its N:
 //     D[128 weight rows][128] (fp32, in TMEM) += W_tile[128][64 k] * [X_hi; X_lo][128][64 k]^T
-// (one MMA of N = 128 per 16 k: columns t and 64 + t of a row are added in the epilogue)
+// (one MMA of N = 128 per 16 k: columns t and 64 + t of a row are added in the epilogue).  Launches over more than 64
+// tokens put up to four token tiles (two with both planes) behind one another in a stage; they form ONE B operand of up
+// to 256 rows, so a k step is still a single MMA (N up to 256) and the weight tile is read once for all of them.  At
+// 256 rows the kernel is no longer bound by HBM but by what an SM can take in: every CTA fetches its own copy of the
+// activation tiles from the L2 (twice the bytes of its weight tile), about 4.7 TB/s over the chip, which caps the
+// contraction near 400 (one plane) to 560 (two planes) TFLOP/s.
 // W tiles come straight from HBM by TMA (128-byte swizzle, evict-first), the two bf16 planes of the split
 // activation come from L2.
 //
@@ -316,6 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         {
             // ---------------- MMA issuer (lane 0 of a convergent warp)
             const uint32_t leader = lane == 0 ? 1u : 0u;
+            const uint32_t idesc_n = RT == 1 ? IDESC : idesc(rt_n * UMMA_N);  // N = all token tiles of this launch
             SegmentIter it(a, blockIdx.x);
             Segment sg;
             int st = 0, j = 0;       // ring stage and its phase, advanced per k block
@@ -337,17 +343,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     }
                     const uint32_t sa = smem_u32(tiles + st * STAGE_BYTES);
                     // the two activation planes of a token tile sit back to back in the stage: one 128-row K-major operand
-                    const uint64_t da = umma_desc(sa);
+                    // and the token tiles of the launch follow one another, so all of them are ONE K-major operand of
+                    // rt_n * UMMA_N rows: a single MMA per k step reads the weight tile once for every token tile, and its
+                    // accumulator columns rt * UMMA_N .. are where the epilogue looks for tile rt
+                    const uint64_t da = umma_desc(sa), db = umma_desc(sa + A_BYTES);
 #pragma unroll
-                    for (int rt = 0; rt < RT; ++rt) {
-                        if (rt < rt_n) {
-                            const uint64_t db = umma_desc(sa + A_BYTES + rt * PL * B_BYTES);
-#pragma unroll
-                            for (int k = 0; k < BK / UMMA_K; ++k) {
-                                const uint64_t adv = (uint64_t)((k * UMMA_K * 2) >> 4);  // 32 bytes per step inside the swizzled row
-                                umma(tmem_d + (uint32_t)(rt * UMMA_N), da + adv, db + adv, IDESC, (i | k) ? 1u : 0u, leader);
-                            }
-                        }
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        const uint64_t adv = (uint64_t)((k * UMMA_K * 2) >> 4);  // 32 bytes per step inside the swizzled row
+                        umma(tmem_d, da + adv, db + adv, idesc_n, (i | k) ? 1u : 0u, leader);
                     }
                     umma_commit(&sm->empty[st], leader);  // frees the stage once these MMAs have read it
                     if (++st == STAGES) {

@@ -15,10 +15,11 @@ from paper_2401_10774_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 CASES = [
-    # name, d, V, K, N (positions: chunks of 256, the last one ragged), weight std
-    ("small_3heads_2chunks", 512, 2048, 3, 300, 0.05),
-    ("small_1chunk_ragged", 256, 1024, 2, 77, 0.05),
-    ("7b_width_1head_2chunks", 4096, 32000, 1, 300, 0.02),
+    # name, d, V, K, N (positions: chunks of up to 1024, a shorter batch is padded to a multiple of 256), weight std
+    ("small_3heads_300", 512, 2048, 3, 300, 0.05),
+    ("small_2heads_77", 256, 1024, 2, 77, 0.05),
+    ("small_2heads_2chunks_1324", 512, 2048, 2, 1324, 0.05),
+    ("7b_width_1head_300", 4096, 32000, 1, 300, 0.02),
 ]
 
 
@@ -70,9 +71,8 @@ def test_heads_loss_and_grads_against_the_oracle(oracle, case):
             report.append("%s[%d] max|err| %.3g of max|g| %.3g, rel. Frobenius %.3g" % (nm, k, float(err.max()), mx, fro))
             assert float(err.max()) <= 2e-2 * mx, report[-1]
             assert fro <= 1e-2, report[-1]
-    chunks = (N + 255) // 256
-    flops = K * chunks * 256 * (4.0 * d * d + 6.0 * V * d)
-    print("%s: loss %s (oracle %s); %s; %.2f ms per call = %.0f TFLOP/s over the padded chunks"
+    flops = K * N * (4.0 * d * d + 6.0 * V * d)
+    print("%s: loss %s (oracle %s); %s; %.2f ms per call = %.0f TFLOP/s"
           % (name, got_loss.round(5).tolist(), np.round(ref["loss_per_head"], 5).tolist(), "; ".join(report), ms, flops / ms / 1e9))
     ctx.close()
 
