@@ -38,7 +38,9 @@ enum {
     MEDUSA_ERR_CACHE_FULL = -4,  /* committing would exceed L_max (nothing is written) */
     MEDUSA_ERR_CUDA = -5,        /* a CUDA runtime call failed */
     MEDUSA_ERR_TIMEOUT = -6,     /* a bounded device-side wait gave up */
-    MEDUSA_ERR_STATE = -7        /* call order: weights/tree not loaded yet */
+    MEDUSA_ERR_STATE = -7,       /* call order: weights/tree not loaded yet */
+    MEDUSA_ERR_NONFINITE = -8,   /* checked build only: a stage produced a NaN or an infinity (device status word) */
+    MEDUSA_ERR_BOUNDS = -9       /* checked build only: a stage produced an index outside its range (device status word) */
 };
 
 enum { MEDUSA_F32 = 0, MEDUSA_BF16 = 1 };
@@ -346,6 +348,14 @@ int32_t medusa_decode_step_batch(medusa_ctx *ctx, const medusa_accept_params *pa
 int32_t medusa_generate(medusa_ctx *ctx, const int32_t *prompt_host, int32_t n_prompt, int32_t G,
                         const medusa_accept_params *params, const float *gumbel_host, int32_t *out_tokens_host,
                         int32_t *emitted_per_step_host, int32_t *steps_host);
+
+/* 1 if this library was built with -DMEDUSA_DEBUG_CHECKS (the "checked" flavour), else 0.  The checked flavour launches,
+ * after the stages of a step, kernels that test what the stage produced -- head logits and backbone logits finite
+ * (MEDUSA_ERR_NONFINITE); tree tokens inside the vocabulary, accepted nodes inside the tree, the chosen row among the
+ * retrieve rows, the next root inside the vocabulary, the cache length inside [0, L_max] (MEDUSA_ERR_BOUNDS) -- and
+ * record the FIRST failure in the device status word (medusa_device_status).  Nothing traps, nothing is skipped, and
+ * the results are those of the default library.  It stands in for a memory checker where none can be run. */
+int32_t medusa_debug_checks_enabled(void);
 
 /* ---- training of the heads with a frozen backbone (paper Sec. 2.2.1, Eq. 1) --------------------------- */
 

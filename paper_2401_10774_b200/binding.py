@@ -55,6 +55,15 @@ class Weights(C.Structure):
 _lib = None
 
 
+def use_checked_library():
+    """Selects the checked flavour of the library (built with `python -m paper_2401_10774_b200.build --debug-checks`):
+    the same entry points, plus device-side validation kernels after the stages of a step.  Call before the first use."""
+    global LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("the CUDA library is already open; choose the flavour before the first call")
+    LIB_PATH = os.path.join(_PKG, "libmedusa_b200_checked.so")
+
+
 def lib():
     """Opens the CUDA library; raises if it is missing (build it with `python -m paper_2401_10774_b200.build`)."""
     global _lib

@@ -1,9 +1,13 @@
 """Builds the CUDA library in-tree with nvcc for sm_100a (cross-compiles without a GPU).
 
-    python -m paper_2401_10774_b200.build [--force] [--verbose] [--timing-aids]
+    python -m paper_2401_10774_b200.build [--force] [--verbose] [--timing-aids] [--debug-checks]
 
 --timing-aids compiles with -DMEDUSA_TIMING_AIDS: only such a build reads the MEDUSA_* environment switches used
 for comparison runs (ring depth, serialised launches, dropped kernel classes); the default build reads none.
+--debug-checks builds a second library, libmedusa_b200_checked.so (-DMEDUSA_DEBUG_CHECKS): after the stages of a step it
+launches small kernels that test what the stage produced (finite logits, token / node / row indices in range, the cache
+length inside the cache) and record MEDUSA_ERR_NONFINITE or MEDUSA_ERR_BOUNDS in the device status word.  Nothing
+traps and nothing is skipped; the default library contains none of these launches.
 """
 from __future__ import annotations
 
@@ -16,6 +20,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libmedusa_b200.so")
+LIB_CHECKED = os.path.join(PKG, "libmedusa_b200_checked.so")
 SOURCES = ["api.cu", "gemm_tc.cu", "simt_kernels.cu", "attention.cu", "attention_flash.cu", "attention_tc.cu", "heads.cu", "posterior.cu", "train_heads.cu", "tree_host.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
@@ -37,21 +42,23 @@ def _newest_header() -> float:
     return t
 
 
-def build_library(force: bool = False, verbose: bool = False, timing_aids: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+def build_library(force: bool = False, verbose: bool = False, timing_aids: bool = False, debug_checks: bool = False) -> str:
+    obj_dir = OBJ + ("_checked" if debug_checks else "")
+    lib_path = LIB_CHECKED if debug_checks else LIB
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
     # a change of flavour rebuilds everything
-    stamp = os.path.join(OBJ, "flavour")
-    flavour = "timing-aids" if timing_aids else "default"
+    stamp = os.path.join(obj_dir, "flavour")
+    flavour = ("timing-aids" if timing_aids else "default") + ("+checks" if debug_checks else "")
     if not os.path.exists(stamp) or open(stamp).read() != flavour:
         force = True
-    extra = ["-DMEDUSA_TIMING_AIDS"] if timing_aids else []
+    extra = (["-DMEDUSA_TIMING_AIDS"] if timing_aids else []) + (["-DMEDUSA_DEBUG_CHECKS"] if debug_checks else [])
     hdr = _newest_header()
     jobs = []
     objs = []
     for src in SOURCES:
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJ, os.path.splitext(src)[0] + ".o")
+        o = os.path.join(obj_dir, os.path.splitext(src)[0] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
             cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-x", "cu", "-c", s, "-o", o]
@@ -66,14 +73,15 @@ def build_library(force: bool = False, verbose: bool = False, timing_aids: bool 
 
     with ThreadPoolExecutor(max_workers=4) as ex:
         list(ex.map(run, jobs))
-    if jobs or not os.path.exists(LIB):
-        tmp = LIB + ".%d.tmp" % os.getpid()
+    if jobs or not os.path.exists(lib_path):
+        tmp = lib_path + ".%d.tmp" % os.getpid()
         run([nvcc, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
-        os.replace(tmp, LIB)
+        os.replace(tmp, lib_path)
     with open(stamp, "w") as f:
         f.write(flavour)
-    return LIB
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv, timing_aids="--timing-aids" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv, timing_aids="--timing-aids" in sys.argv,
+                        debug_checks="--debug-checks" in sys.argv))

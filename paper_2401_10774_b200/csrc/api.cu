@@ -197,6 +197,38 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 __global__ void set_i32_kernel(int32_t *p, int32_t v) {
     pdl_enter(); *p = v; }
 
+// ---- the checked flavour (-DMEDUSA_DEBUG_CHECKS): validation kernels launched after the stages of a step.  They only
+// read what the stage produced and record the first failure in the device status word; nothing traps or is skipped.
+#ifdef MEDUSA_DEBUG_CHECKS
+__global__ void __launch_bounds__(256) debug_finite_kernel(const float *__restrict__ p, size_t n, int32_t *status)
+{
+    bool bad = false;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        bad |= !isfinite(p[i]);
+    if (bad) atomicCAS(status, MEDUSA_OK, MEDUSA_ERR_NONFINITE);
+}
+__global__ void __launch_bounds__(256) debug_range_kernel(const int32_t *__restrict__ p, int n, int lo, int hi, int32_t *status)
+{
+    bool bad = false;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        bad |= p[i] < lo || p[i] > hi;
+    if (bad) atomicCAS(status, MEDUSA_OK, MEDUSA_ERR_BOUNDS);
+}
+void debug_finite(medusa_ctx *c, const float *p, size_t n)
+{
+    if (n) debug_finite_kernel<<<(unsigned)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, c->stream>>>(p, n, c->d_state + ST_STATUS);
+}
+void debug_range(medusa_ctx *c, const int32_t *p, int n, int lo, int hi)
+{
+    if (n > 0) debug_range_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(p, n, lo, hi, c->d_state + ST_STATUS);
+}
+#define DEBUG_FINITE(c, p, n) debug_finite(c, p, n)
+#define DEBUG_RANGE(c, p, n, lo, hi) debug_range(c, p, n, lo, hi)
+#else
+#define DEBUG_FINITE(c, p, n) ((void)0)
+#define DEBUG_RANGE(c, p, n, lo, hi) ((void)0)
+#endif
+
 constexpr int ATTN_TC_MIN_L = 2048;  // measured crossover of the two attention kernels at T = 64, 32 heads
 
 enum { PC_GEMM = 0, PC_ATTENTION = 1, PC_HEADS = 2, PC_ELEMWISE = 3, PC_TOPK = 4, PC_POSTERIOR = 5, PC_COMMIT = 6 };
@@ -343,6 +375,10 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
     cudaStream_t s = c->stream;
     const int T = n_seq > 1 ? n_seq * TREE_ROWS : T_seq;  // rows of the pass
     int32_t *cache_len = c->d_state + ST_CACHE_LEN;
+    for (int b = 0; b < n_seq; ++b) {  // (checked flavour) the pass's tokens and every sequence's cache length
+        DEBUG_RANGE(c, tokens + (size_t)b * TREE_ROWS, T_seq, 0, m.vocab - 1);
+        DEBUG_RANGE(c, n_seq > 1 ? c->state_all + (size_t)b * ST_WORDS + ST_CACHE_LEN : cache_len, 1, 0, m.L_max);
+    }
     PROF(c, PC_ELEMWISE, 1, launch_embed(dt, tokens, c->w.embed, c->x, T, d, m.vocab, s));
     if (n_seq > 1) {
         for (int b = 0; b < n_seq; ++b)
@@ -442,6 +478,10 @@ int32_t tree_pass(medusa_ctx *c, const int32_t *tokens, int T_seq, const uint64_
     PlaneDesc pd{};
     TRY(project(c, c->hidden, &c->map_hidden, wl, c->use_tc ? &c->map_lm : nullptr, 1, m.vocab, d, c->logits, 0, m.vocab, T,
                 lm_row0, true, &pd));
+    for (int b = 0; b < n_seq; ++b) {  // (checked flavour) the logits of every row that holds a token
+        const int r0 = b * TREE_ROWS + (b == 0 ? lm_row0 : 0), r1 = b * TREE_ROWS + T_seq;
+        if (r1 > r0) DEBUG_FINITE(c, c->logits + (size_t)r0 * m.vocab, (size_t)(r1 - r0) * m.vocab);
+    }
     return MEDUSA_OK;
 }
 
@@ -625,6 +665,15 @@ extern "C" int32_t medusa_destroy(medusa_ctx *c)
     if (c->own_stream) cudaStreamDestroy(c->stream);
     delete c;
     return MEDUSA_OK;
+}
+
+extern "C" int32_t medusa_debug_checks_enabled(void)
+{
+#ifdef MEDUSA_DEBUG_CHECKS
+    return 1;
+#else
+    return 0;
+#endif
 }
 
 extern "C" const char *medusa_last_error(const medusa_ctx *c) { return c ? c->err.c_str() : "null context"; }
@@ -866,6 +915,8 @@ static int32_t heads_impl(medusa_ctx *c, const void *h, int h_is_f32, const void
              launch_topk(z, K, c->m.vocab, c->tree.topk, topk_idx, topk_val, c->topk_scratch, c->stream));
     }
     PROF(c, PC_TOPK,1, launch_expand(root_token, topk_idx, c->d_tree_idx, tree_tok, c->tree.T, c->stream));
+    if (K > 0) DEBUG_FINITE(c, z, (size_t)K * c->m.vocab);
+    DEBUG_RANGE(c, tree_tok, c->tree.T, 0, c->m.vocab - 1);
     MEDUSA_LAUNCH_CHECK(c);
     return MEDUSA_OK;
 }
@@ -888,6 +939,7 @@ extern "C" int32_t medusa_tree_attention(medusa_ctx *c, const void *q, const voi
     if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
         return fail(c, MEDUSA_ERR_INVALID_ARG, "medusa_tree_attention: tensors must be 16-byte aligned");
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
+    DEBUG_RANGE(c, cache_len, 1, 0, c->m.L_max);
     const medusa_model_desc &m = c->m;
     const int T = c->tree.T;
     const void *qq = q, *kk = k_new;
@@ -937,6 +989,10 @@ extern "C" int32_t medusa_evaluate_posterior(medusa_ctx *c, const float *logits,
     a.node_part = c->node_part; a.stat_slices = NODE_STAT_SLICES;
     a.best = best; a.accept_len = accept_len; a.next_root = next_root; a.acc_nodes = acc_nodes;
     PROF(c, PC_POSTERIOR,2, launch_evaluate_posterior(a, c->stream));
+    DEBUG_RANGE(c, acc_nodes, c->tree.depth + 1, -1, c->tree.T - 1);
+    DEBUG_RANGE(c, best, 1, 0, c->tree.P - 1);
+    DEBUG_RANGE(c, accept_len, 1, 0, c->tree.depth);
+    DEBUG_RANGE(c, next_root, 1, 0, c->m.vocab - 1);
     MEDUSA_LAUNCH_CHECK(c);
     return MEDUSA_OK;
 }

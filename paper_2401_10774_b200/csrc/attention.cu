@@ -24,7 +24,7 @@ tree_attention_simt_kernel(const AT *__restrict__ q, const AT *__restrict__ k_ne
     if (i >= T)
         return;
     const int hk = h / (H / Hkv);  // grouped-query attention: the key/value head this query head reads
-    const int L = *cache_len;
+    const int L = min(max(*cache_len, 0), L_max);  // a length outside [0, L_max] would index past the caches
     const float scale = rsqrtf((float)D);
     float qv[E], o[E];
 #pragma unroll
