@@ -338,7 +338,9 @@ int32_t medusa_select_sequence(medusa_ctx *ctx, int32_t b);
  * commit run per sequence exactly as in medusa_decode_step (same acceptance rule for all).  The uploaded tree must have
  * at most 64 nodes (SHAPE otherwise).  gumbel (nullable): float [B][V] device noise rows ([B][V + T] for REJECTION); emitted_host [B][depth+1] and
  * n_emitted_host [B] (nullable, pinned host memory recommended): async copies, valid after the stream is synchronised.
- * Every sequence must have been prefilled.  The step is enqueued directly (no whole-step graph). */
+ * Every sequence must have been prefilled.  Like medusa_decode_step, the second consecutive batched step with the same
+ * launch configuration is captured into a CUDA graph and replayed afterwards (the noise rows are staged through a
+ * buffer of the context). */
 int32_t medusa_decode_step_batch(medusa_ctx *ctx, const medusa_accept_params *params, const float *gumbel,
                                  int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host);
 

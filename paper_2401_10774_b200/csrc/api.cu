@@ -1171,6 +1171,9 @@ constexpr size_t MAX_STEP_GRAPHS = 16;
 // Captures one step with key `key` from the stream and instantiates it.  Nothing runs during the capture; on any
 // failure the capture is closed, step graphs are switched off for this context and false is returned (the caller
 // then enqueues the step directly).
+static int32_t decode_step_batch_launches(medusa_ctx *c, const medusa_accept_params *params, const float *gumbel,
+                                          int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host);
+
 static bool capture_step_graph(medusa_ctx *c, const medusa_ctx::StepKey &key, const medusa_accept_params *params,
                                const float *gumbel)
 {
@@ -1181,7 +1184,9 @@ static bool capture_step_graph(medusa_ctx *c, const medusa_ctx::StepKey &key, co
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
     if (ok) {
-        const int32_t rc = decode_step_launches(c, params, gumbel, key.max_commit, key.emitted_host, key.n_emitted_host);
+        const int32_t rc = key.seq < 0  // a batched step (all sequences) or the selected sequence's step
+                               ? decode_step_batch_launches(c, params, gumbel, key.max_commit, key.emitted_host, key.n_emitted_host)
+                               : decode_step_launches(c, params, gumbel, key.max_commit, key.emitted_host, key.n_emitted_host);
         const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
         ok = rc == MEDUSA_OK && e == cudaSuccess && graph != nullptr;
     }
@@ -1293,11 +1298,63 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
     if (c->tree.T > TREE_ROWS)
         return fail(c, MEDUSA_ERR_SHAPE, "a batched step gives every sequence one tile of 64 token rows: the tree has %d nodes", c->tree.T);
     const medusa_model_desc &m = c->m;
-    const int B = c->B, depth1 = c->tree.depth + 1, T = c->tree.T;
+    const int B = c->B, depth1 = c->tree.depth + 1;
     if (max_commit > depth1) max_commit = depth1;
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
     const int keep = c->cur;
     c->L_upper_all[keep] = c->L_upper;
+
+    // The launches of a batched step depend on the host through the same values as a single step's (acceptance parameters,
+    // commit budget, presence of noise, the host result pointers): the second consecutive batched step with the same key
+    // is captured into a graph (sequence index -1 in the key) and replayed afterwards.
+    bool graphed = false;
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (c->step_graphs_on && !c->prof && c->skip_mask == 0 && c->withhold == 0 &&
+        cudaStreamIsCapturing(c->stream, &capturing) == cudaSuccess && capturing == cudaStreamCaptureStatusNone) {
+        medusa_ctx::StepKey key;
+        memset(&key, 0, sizeof key);
+        key.max_commit = max_commit;
+        key.seq = -1;
+        const bool noisy = gumbel && mode_reads_noise(params);
+        key.has_gumbel = noisy ? 1 : 0;
+        key.p = *params;
+        key.emitted_host = emitted_host;
+        key.n_emitted_host = n_emitted_host;
+        medusa_ctx::StepGraph *g = nullptr;
+        for (auto &cand : c->step_graphs)
+            if (memcmp(&cand.key, &key, sizeof key) == 0) g = &cand;
+        if (!g && c->have_last_key && memcmp(&c->last_key, &key, sizeof key) == 0 && graph_safe_host_ptr(emitted_host) &&
+            graph_safe_host_ptr(n_emitted_host) && capture_step_graph(c, key, params, noisy ? c->gumbel_all : nullptr))
+            g = &c->step_graphs.back();
+        c->last_key = key;
+        c->have_last_key = true;
+        if (g) {
+            // the graph reads the sequences' noise rows from the context's own buffer, packed [B][row]
+            if (noisy && gumbel != c->gumbel_all)
+                MEDUSA_CUDA(c, cudaMemcpyAsync(c->gumbel_all, gumbel, (size_t)B * noise_floats(c, params->mode) * sizeof(float),
+                                               cudaMemcpyDeviceToDevice, c->stream));
+            MEDUSA_CUDA(c, cudaGraphLaunch(g->exec, c->stream));
+            for (int i = 0; i < MEDUSA_PROF_CATEGORIES; ++i) c->launches[i] += g->launches[i];
+            g->used = ++c->step_clock;
+            graphed = true;
+        }
+    }
+    int32_t rc = MEDUSA_OK;
+    if (!graphed) rc = decode_step_batch_launches(c, params, gumbel, max_commit, emitted_host, n_emitted_host);
+    for (int b = 0; b < B; ++b) {
+        const int up = c->L_upper_all[b] + max_commit;
+        c->L_upper_all[b] = up > m.L_max ? m.L_max : up;
+    }
+    point_at(c, keep);
+    return rc;
+}
+
+// The launches of one batched step (also what a capture records).  Leaves the selected-sequence views on the last sequence.
+static int32_t decode_step_batch_launches(medusa_ctx *c, const medusa_accept_params *params, const float *gumbel,
+                                          int32_t max_commit, int32_t *emitted_host, int32_t *n_emitted_host)
+{
+    const medusa_model_desc &m = c->m;
+    const int B = c->B, depth1 = c->tree.depth + 1, T = c->tree.T;
     int32_t rc = MEDUSA_OK;
     // (1) candidates of every sequence: the heads of all sequences in two launches (every head weight is read once),
     // then top-k and the sequence's tile of tree tokens per sequence
@@ -1353,10 +1410,7 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
         if (n_emitted_host &&
             cudaMemcpyAsync(n_emitted_host + b, st + ST_N_EMITTED, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
             rc = fail(c, MEDUSA_ERR_CUDA, "copy of the emitted count failed");
-        int up = c->L_upper_all[b] + max_commit;
-        c->L_upper_all[b] = up > m.L_max ? m.L_max : up;
     }
-    point_at(c, keep);
     return rc;
 }
 

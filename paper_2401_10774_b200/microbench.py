@@ -8,6 +8,10 @@ the L2), prefills a seeded prompt and runs a few tree-verification steps through
 under a profiler restricted to one kernel; prints per-category device times from the library's own events.
 `--attention L` times the stand-alone `tree_attention` entry instead: `--caches` launches over that many distinct
 K/V caches of length L (together larger than the L2) per repetition, replayed from a CUDA graph.
+`--heads-train N` times the forward/backward pass of the heads' training objective over N positions (one head unless
+`--heads K`), and reports it against the measured dense bf16 throughput.
+
+    python -m paper_2401_10774_b200.microbench --heads-train 4096 [--model 7b] [--heads 1] [--steps 3]
 """
 from __future__ import annotations
 
@@ -41,9 +45,13 @@ def main():
     ap.add_argument("--device-weights", action="store_true",
                     help="draw the weights on the device (N(0, 0.02^2), not the seeded host recipe): seconds instead of a "
                          "minute of set-up, for timing runs whose numbers do not depend on the values")
+    ap.add_argument("--heads-train", type=int, default=0, metavar="N", help="time the heads' training pass over N positions")
+    ap.add_argument("--heads", type=int, default=1, help="heads in the training pass")
     args = ap.parse_args()
     if args.attention:
         return attention_only(args)
+    if args.heads_train:
+        return heads_train_only(args)
 
     cfg = I.model_shape(args.model, n_layers=args.layers)
     tree_name = args.tree or ("sparse64_d5" if cfg["n_medusa"] >= 5 else "sparse64_d4")
@@ -157,6 +165,44 @@ def attention_only(args):
     print(json.dumps(dict(op="tree_attention", model=args.model, L=L, T=T, H=H, us_per_launch=round(us, 2),
                           achieved_gbs=round(nbytes / us / 1e3, 1), frac=round(nbytes / us / 1e3 / peak, 3), peak_gbs=peak,
                           peak_source=src, status=ctx.device_status())))
+    ctx.close()
+
+
+def heads_train_only(args):
+    import torch
+
+    from . import binding as B
+    from . import inputs as I
+    from . import roofline as R
+
+    shape = I.model_shape(args.model, n_layers=0)
+    d, V, K, N = shape["d"], shape["vocab"], args.heads, args.heads_train
+    cfg = dict(n_layers=0, d=d, n_heads=shape["n_heads"], head_dim=shape["head_dim"], ffn=8, vocab=V, n_medusa=K)
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    rnd = lambda *sh: (torch.randn(*sh, device="cuda", generator=gen) * 0.02).bfloat16()
+    w = dict(embed=rnd(V, d), lm_head=rnd(V, d), final_norm=torch.ones(d, device="cuda").bfloat16(), layers=[],
+             medusa_w1=rnd(K, d, d), medusa_w2=rnd(K, V, d))
+    ctx = B.Context(cfg, B.BF16, 64)
+    ctx.load_weights(w)
+    h = torch.randn(N, d, device="cuda", generator=gen).bfloat16()
+    y = torch.randint(0, V, (K, N), device="cuda", dtype=torch.int32)
+    loss = torch.zeros(K + 1, device="cuda")
+    g1, g2 = torch.zeros(K, d, d, device="cuda"), torch.zeros(K, V, d, device="cuda")
+    for _ in range(max(args.warmup, 1)):
+        ctx.heads_loss_and_grads(h, y, loss, g1, g2)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.heads_loss_and_grads(h, y, loss, g1, g2)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    flop = K * N * (4.0 * d * d + 6.0 * V * d)  # five projections per head and position
+    peak, src = R.tensor_peak_tflops()
+    print(json.dumps(dict(op="heads_loss_and_grads", model=args.model, heads=K, positions=N, ms_per_pass=round(ms, 3),
+                          positions_per_s=round(N / ms * 1e3), tflops=round(flop / ms / 1e9, 1), frac=round(flop / ms / 1e9 / peak, 3),
+                          peak_tflops=peak, peak_source=src, loss=[round(float(v), 4) for v in loss.cpu()], status=ctx.device_status())))
     ctx.close()
 
 

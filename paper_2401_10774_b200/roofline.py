@@ -84,6 +84,18 @@ def hbm_peak_gbs():
     return 6650.0, "fallback"
 
 
+def tensor_peak_tflops():
+    """(TFLOP/s, source): the measured dense bf16 throughput (a burst of a library GEMM) recorded beside the package, else
+    the fallback."""
+    import json
+    import os
+
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
 # ---- DRAM traffic taken from profiler captures ----
 # A capture describes the kernel source it was taken from: the figure is reported only while the SHA-256 of that
 # source file still equals the one recorded with the capture, so a changed kernel never inherits an old number.
