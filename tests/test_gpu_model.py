@@ -284,6 +284,50 @@ def test_tiny_fp32_typical_sampled_generate_matches_oracle(oracle):
     ctx.close()
 
 
+def test_tiny_fp32_rejection_sampling_generate_matches_an_oracle_loop(oracle):
+    """Rejection sampling through the convenience loop (host noise rows of V + T floats per step) on the tiny fp32 model
+    with sharpened heads: the token stream equals a loop over the oracle's stage functions fed the same noise."""
+    torch, B, U = _gpu()
+    cfg = I.model_shape("tiny")
+    ctx, om, ot = _setup(oracle, cfg, "f32", "dense22", 160, seed=0, head_init="lm_copy")
+    V, T, K = cfg["vocab"], ot["T"], ot["depth"]
+    prompt = I.make_prompt(32, V, 1)
+    G, tau = 40, 0.05   # a low temperature sharpens the random-init distributions, so that candidates do get accepted
+    f32 = lambda x: float(np.float32(x))
+    noise = np.concatenate([I.gumbel_noise(G, V, 54), I.uniform_noise(G, T, 55)], axis=1)
+    got = ctx.generate(prompt, G, B.AcceptParams(mode=B.REJECTION, temperature=tau), gumbel_host=noise)
+    # the same loop over the oracle's stages
+    kc = np.zeros(om.cache_shape(160)); vc = np.zeros_like(kc)
+    last = oracle.tree_pass(om, prompt, oracle.chain_tree(len(prompt)), 0, kc, vc)
+    oracle.accept_and_update_kv(last["tree_k"], last["tree_v"], kc, vc, np.arange(len(prompt)), len(prompt) - 1, len(prompt), 0,
+                                last["hidden"], prompt)
+    L, h_last, root = len(prompt), last["hidden"][-1].copy(), int(oracle.topk(last["logits"][-1].astype(np.float32), 1)[0])
+    out, per_step, step, min_margin = [], [], 0, np.inf
+    while len(out) < G:
+        _, z = oracle.medusa_heads(h_last, om.w["medusa_w1"][:K], om.w["medusa_w2"][:K])
+        ti = np.stack([oracle.topk(z[k].astype(np.float32), ot["topk"]) for k in range(K)])
+        tok = oracle.expand_candidates(root, ti, ot)[0]
+        p = oracle.tree_pass(om, tok, ot, L, kc, vc)
+        r = oracle.evaluate_posterior(p["logits"].astype(np.float32), tok, ot, mode=oracle.REJECTION, tau=f32(tau),
+                                      gumbel=noise[step, :V], uniform=noise[step, V:])
+        min_margin = min(min_margin, r["min_margin"])
+        c = oracle.accept_and_update_kv(p["tree_k"], p["tree_v"], kc, vc, r["acc_nodes"], r["accept_len"], G - len(out), L,
+                                        p["hidden"], tok)
+        em = [int(t) for t in c["emitted"] if t >= 0]
+        n = len(em)
+        # a budget that cuts the accepted path short makes the path's next token the next root (as the library does)
+        root = int(tok[r["acc_nodes"][n]]) if n < 1 + r["accept_len"] else r["next_root"]
+        L, h_last = c["L"], c["h_last"]
+        out += em
+        per_step.append(n)
+        step += 1
+    assert min_margin > 2e-3, "a uniform too close to its acceptance probability for a float32-vs-double comparison: change the seed"
+    assert got["tokens"].tolist() == out[:G]
+    assert got["emitted_per_step"].tolist() == per_step
+    assert max(per_step) > 1, "the sharpened distributions must let some candidates through"
+    ctx.close()
+
+
 @pytest.mark.parametrize("mode", ["greedy", "typical_gumbel"])
 def test_step_graph_replay_matches_plain_launches(oracle, mode):
     # The library captures a decode step into a CUDA graph on the second use of a launch configuration.  The same
