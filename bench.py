@@ -283,6 +283,7 @@ def run_gpu(args):
     tree = ctx.build_tree_buffers(B.default_tree_paths(spec["per_depth_topk"], spec["n_nodes"]))
     if args.planes != 2:
         ctx.set_option(B.OPT_ACTIVATION_PLANES, args.planes)
+    ctx.set_option(B.OPT_PACK_WEIGHTS, args.pack_weights)  # read by load_weights below
     ctx.load_weights(dw)
     for b in range(NB):
         ctx.select_sequence(b)
@@ -445,7 +446,7 @@ def run_gpu(args):
             "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": WORKLOAD["name"], "tree_nodes": T, "prompt": WORKLOAD["prompt"], "L_max": WORKLOAD["L_max"],
-                       "cache_len_start": L0 // NB, "heads": cfg["n_medusa"], "replicas": world, "batch": NB, "activation_planes": args.planes,
+                       "cache_len_start": L0 // NB, "heads": cfg["n_medusa"], "replicas": world, "batch": NB, "activation_planes": args.planes, "packed_weights": bool(args.pack_weights),
                        "l2": "inputs larger than L2: every step streams %.1f GB of weights" % (sb["gemm_weights"] / 1e9)},
             "clocks": clocks,
             "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": "tokens/s",
@@ -507,6 +508,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS), help="7b: the headline configuration")
+    ap.add_argument("--pack-weights", type=int, default=1, choices=(0, 1),
+                    help="1 (the library's default): the context streams its own tile-by-tile copy of the backbone matrices; "
+                         "0: the row-major tensors as given")
     ap.add_argument("--planes", type=int, default=2, choices=(1, 2),
                     help="activation planes the projections read (2: hi + lo, the default and the headline; 1: hi only)")
     args = ap.parse_args()

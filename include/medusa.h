@@ -144,10 +144,16 @@ enum {
                                       * next tcgen05 attention launch, one CTA's producer issues no load at all, so that its
                                       * consumers' bounded waits expire with nothing in flight; the launch returns, its output
                                       * is unusable and the device status becomes MEDUSA_ERR_TIMEOUT */
-    MEDUSA_OPT_ACTIVATION_PLANES = 6  /* bf16 model: planes of every activation the projections read.  2 (default): a value
+    MEDUSA_OPT_ACTIVATION_PLANES = 6, /* bf16 model: planes of every activation the projections read.  2 (default): a value
                                        * y is held as hi = bf16(y) and lo = bf16(y - hi) and a projection is W hi + W lo
                                        * (accurate to ~2^-17); 1: hi only -- half the tensor-core work and up to 256 token
                                        * rows per weight stream (large trees, batches), at bf16 accuracy of the inputs */
+    MEDUSA_OPT_PACK_WEIGHTS = 7        /* bf16 model, read by medusa_load_weights: 1 (default) = the context keeps its own
+                                       * copy of the backbone matrices and the LM head, re-laid tile by tile so that the
+                                       * 16 KiB a CTA requests per k block are consecutive bytes (costs the size of those
+                                       * weights in device memory a second time; same arithmetic, bit-identical results,
+                                       * the projections about 3.5 % faster); 0 = the projections stream the caller's
+                                       * row-major tensors and nothing is copied */
 };
 
 /* ---- lifetime ------------------------------------------------------------------------------------ */

@@ -20,7 +20,7 @@ GREEDY, TYPICAL, REJECTION = 0, 1, 2  # REJECTION: the noise row is gumbel[V] fo
 (WS_LOGITS, WS_HIDDEN, WS_TREE_K, WS_TREE_V, WS_K_CACHE, WS_V_CACHE, WS_HEAD_LOGITS, WS_TOPK_IDX, WS_TREE_TOK,
  WS_ACC_NODES, WS_STATE, WS_H_LAST, WS_EMITTED, WS_TAP_X_IN, WS_TAP_X_OUT, WS_TAP_ATT, WS_TAP_XN_OUT) = range(17)
 (OPT_STEP_GRAPHS, OPT_ATTENTION_KERNEL, OPT_ATTENTION_LENGTH_HINT, OPT_LAYER_TAP, OPT_SPIN_LIMIT,
- OPT_WITHHOLD_LOAD, OPT_ACTIVATION_PLANES) = range(7)
+ OPT_WITHHOLD_LOAD, OPT_ACTIVATION_PLANES, OPT_PACK_WEIGHTS) = range(8)
 LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 

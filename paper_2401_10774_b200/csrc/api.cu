@@ -83,6 +83,8 @@ struct medusa_ctx {
     std::vector<TensorMap> wmaps;  // per layer: wq, wk, wv, wo, w_gate, w_up, w_down
     // activation planes the projections read (MEDUSA_OPT_ACTIVATION_PLANES): 2 = hi + lo (default), 1 = hi only
     int act_planes = 2;
+    // MEDUSA_OPT_PACK_WEIGHTS: the weight maps describe the context's own packed copies (packed_on: as loaded)
+    bool pack_weights = true, packed_on = false;
     // the lo plane of a split activation (null in the f32 model and when the projections read one plane only)
     void *lo(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 && act_planes == 2 ? (char *)hi + (size_t)rows * width * 2 : nullptr; }
     // the second plane of q, which the attention kernel reads whatever the projections do
@@ -342,7 +344,8 @@ int32_t project(medusa_ctx *c, const void *X, const TensorMap *mapX, const void 
             if (wh) c->withhold = 0;
             const int Tt = T - r0 < rows_per_launch ? T - r0 : rows_per_launch, row0t = row0 > r0 ? row0 - r0 : 0;
             PROF(c, PC_GEMM, 1, e = launch_gemm_tc(mapX, maps, n_seg, seg_cols, K, *pd, P + (size_t)r0 * ldy, ldy, Tt, row0t,
-                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0, RT, c->act_planes));
+                                                   c->d_state + ST_STATUS, c->stream, seg0_cols, c->spin_limit, wh, r0, c->rows + r0, RT, c->act_planes, false, 0, 0,
+                                                   c->packed_on));
             if (e != cudaSuccess) return fail(c, MEDUSA_ERR_CUDA, "tensor-core GEMM launch failed: %s", cudaGetErrorString(e));
         }
         return MEDUSA_OK;
@@ -774,6 +777,10 @@ extern "C" int32_t medusa_set_option(medusa_ctx *c, int32_t option, int64_t valu
         drop_step_graphs(c);
         c->act_planes = (int)value;
         return MEDUSA_OK;
+    case MEDUSA_OPT_PACK_WEIGHTS:
+        if (value != 0 && value != 1) return fail(c, MEDUSA_ERR_INVALID_ARG, "pack weights: 0 or 1");
+        c->pack_weights = value == 1;  // takes effect with the next medusa_load_weights
+        return MEDUSA_OK;
     case MEDUSA_OPT_WITHHOLD_LOAD:
         if (value < 0 || value > 2) return fail(c, MEDUSA_ERR_INVALID_ARG, "withhold: 0 (off), 1 (next tensor-core GEMM) or 2 (next tcgen05 attention)");
         c->withhold = (int)value;
@@ -1054,15 +1061,33 @@ extern "C" int32_t medusa_load_weights(medusa_ctx *c, const medusa_weights *w)
     if (c->use_tc) {
         const int d = m.d, HD = m.n_heads * m.head_dim, HkvD = c->Hkv * m.head_dim, F = m.ffn;
         c->wmaps.resize((size_t)m.n_layers * 7);
-        bool ok = make_weight_map(&c->map_lm, w->lm_head, m.vocab, d);
+        c->packed_on = c->pack_weights;
+        bool ok = true;
+        // one matrix: its map over the caller's tensor, or a packed copy of it (kept by the context) and that copy's map
+        auto add = [&](TensorMap *tm, const void *W, int N, int K) -> int32_t {
+            if (!c->packed_on) {
+                ok = ok && make_weight_map(tm, W, N, K);
+                return MEDUSA_OK;
+            }
+            void *Wp = nullptr;
+            TRY(dev_alloc_bytes(c, &Wp, packed_weight_elems(N, K) * 2));
+            launch_pack_weight(W, N, K, Wp, c->stream);
+            ok = ok && make_packed_weight_map(tm, Wp, N, K);
+            return MEDUSA_OK;
+        };
+        TRY(add(&c->map_lm, w->lm_head, m.vocab, d));
         for (int l = 0; l < m.n_layers && ok; ++l) {
             const void *const *lw = c->layers.data() + (size_t)l * 9;
             TensorMap *wm = c->wmaps.data() + (size_t)l * 7;
-            ok = make_weight_map(wm + 0, lw[1], HD, d) && make_weight_map(wm + 1, lw[2], HkvD, d) &&
-                 make_weight_map(wm + 2, lw[3], HkvD, d) && make_weight_map(wm + 3, lw[4], d, HD) &&
-                 make_weight_map(wm + 4, lw[6], F, d) && make_weight_map(wm + 5, lw[7], F, d) &&
-                 make_weight_map(wm + 6, lw[8], d, F);
+            TRY(add(wm + 0, lw[1], HD, d));
+            TRY(add(wm + 1, lw[2], HkvD, d));
+            TRY(add(wm + 2, lw[3], HkvD, d));
+            TRY(add(wm + 3, lw[4], d, HD));
+            TRY(add(wm + 4, lw[6], F, d));
+            TRY(add(wm + 5, lw[7], F, d));
+            TRY(add(wm + 6, lw[8], d, F));
         }
+        MEDUSA_LAUNCH_CHECK(c);
         if (!ok) return fail(c, MEDUSA_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
     }
     c->have_weights = true;

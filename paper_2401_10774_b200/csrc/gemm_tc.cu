@@ -299,7 +299,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     uint8_t *st = tiles + s * STAGE_BYTES;
                     const int k = (sg.kb0 + i) * BK;
                     mbar_expect_tx(&sm->full[s], stage_tx);
-                    tma_load_2d(st, mapW, k, trow, &sm->full[s], pol_stream);
+                    // packed weights: tile (tile row, k block) is 16 KiB of consecutive bytes, rows of 64 elements
+                    if (a.packed)
+                        tma_load_2d(st, mapW, 0, ((trow >> 7) * a.KB + (sg.kb0 + i)) * BM, &sm->full[s], pol_stream);
+                    else
+                        tma_load_2d(st, mapW, k, trow, &sm->full[s], pol_stream);
                     if (waited) {
                         load_x(st, k, &sm->full[s]);
                     } else {
@@ -504,6 +508,36 @@ bool make_tensor_map(TensorMap *out, const void *base, int rows, int K, int box_
 static_assert(sizeof(TensorMap) == sizeof(CUtensorMap), "TensorMap must mirror CUtensorMap");
 
 bool make_weight_map(TensorMap *out, const void *W, int N, int K) { return make_tensor_map(out, W, N, K, BM); }
+bool make_packed_weight_map(TensorMap *out, const void *Wp, int N, int K)
+{
+    const long long tiles = (N + BM - 1) / BM, KB = (K + BK - 1) / BK;
+    if (tiles * KB * BM > 0x7fffffffLL) return false;
+    return make_tensor_map(out, Wp, (int)(tiles * KB * BM), BK, BM);
+}
+size_t packed_weight_elems(int N, int K) { return (size_t)((N + BM - 1) / BM) * ((K + BK - 1) / BK) * BM * BK; }
+
+// Wp[((tile row * KB + k block) * 128 + r) * 64 + c] = W[(tile row * 128 + r) * K + k block * 64 + c], zero outside W:
+// one block per (k block, tile row), 16 bytes per thread
+__global__ void __launch_bounds__(1024) pack_weight_kernel(const bf16 *__restrict__ W, int N, int K, bf16 *__restrict__ Wp)
+{
+    const int kb = blockIdx.x, tr = blockIdx.y, KB = gridDim.x;
+    const int r = threadIdx.x >> 3, c8 = threadIdx.x & 7;
+    const int row = tr * BM + r, col = kb * BK + c8 * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < N && col + 8 <= K) {
+        v = *reinterpret_cast<const uint4 *>(W + (size_t)row * K + col);
+    } else if (row < N && col < K) {  // a ragged last k block: element by element
+        bf16 t[8];
+        for (int e = 0; e < 8; ++e)
+            t[e] = col + e < K ? W[(size_t)row * K + col + e] : __float2bfloat16_rn(0.f);
+        v = *reinterpret_cast<const uint4 *>(t);
+    }
+    *reinterpret_cast<uint4 *>(Wp + (((size_t)tr * KB + kb) * BM + r) * BK + c8 * 8) = v;
+}
+void launch_pack_weight(const void *W, int N, int K, void *Wp, cudaStream_t s)
+{
+    pack_weight_kernel<<<dim3((K + BK - 1) / BK, (N + BM - 1) / BM), 1024, 0, s>>>((const bf16 *)W, N, K, (bf16 *)Wp);
+}
 bool make_act_map(TensorMap *out, const void *X_planes, int K, int rows) { return make_tensor_map(out, X_planes, 2 * rows, K, BN); }
 
 // CTAs resident per SM and TMA ring depth; MEDUSA_GEMM_CTAS_PER_SM / MEDUSA_GEMM_STAGES override for tuning
@@ -584,7 +618,7 @@ static GemmKernel gemm_kernel_transposing()
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
                            int seg0_cols, uint32_t spin_limit, int withhold, int x_row_hi, int x_row_lo, int row_tiles,
-                           int planes, bool serialize, int out_t, long long ldt)
+                           int planes, bool serialize, int out_t, long long ldt, bool packed)
 {
     if (out_t && (pd.G != 0 || row_tiles < 4 || planes != 1))
         return cudaErrorInvalidValue;  // a transposed result needs whole tiles (one plane, every element written once);
@@ -628,6 +662,7 @@ cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, 
     a.x_row_lo = x_row_lo;
     a.out_t = out_t;
     a.ldt = ldt;
+    a.packed = packed ? 1 : 0;
     const CUtensorMap *w0 = (const CUtensorMap *)mapW[0];
     const CUtensorMap *w1 = (const CUtensorMap *)mapW[n_seg > 1 ? 1 : 0];
     const CUtensorMap *w2 = (const CUtensorMap *)mapW[n_seg > 2 ? 2 : 0];

@@ -54,12 +54,20 @@ struct GemmTcArgs {
     uint32_t spin_limit;     // polls before a bounded wait gives up
     int withhold;            // test hook: CTA 0's producer issues no load at all, so its consumers' waits expire
     int x_row_hi, x_row_lo;  // rows of the activation tensor where this launch's 64 token rows start in the hi / lo plane
+    int packed;              // 1: the weight maps describe packed matrices (make_packed_weight_map)
     int out_t;               // 0: P[t][n];  1: P[n * ldt + t] = result (transposed store);  2: P[n * ldt + t] += result
     long long ldt;           // row stride of the transposed output (whole-tile launches only)
 };
 
 // W: [N][K] bf16 row-major
 bool make_weight_map(TensorMap *out, const void *W, int N, int K);
+// Packed weights: the matrix re-laid tile by tile, [ceil(N/128)][ceil(K/64)][128 rows][64 k], zero-padded, so that the
+// 16 KiB a CTA requests per k block are consecutive bytes (a row-major matrix hands out 128 separate 128-byte pieces
+// K * 2 bytes apart, which the memory system serves less efficiently).  launch_pack_weight writes that layout,
+// make_packed_weight_map describes it, launch_gemm_tc(..., packed = true) addresses it.
+size_t packed_weight_elems(int N, int K);
+void launch_pack_weight(const void *W, int N, int K, void *Wp, cudaStream_t s);
+bool make_packed_weight_map(TensorMap *out, const void *Wp, int N, int K);
 // X_planes: split activation, [2][rows][K] bf16 (hi plane, then lo plane; rows a multiple of 64)
 bool make_act_map(TensorMap *out, const void *X_planes, int K, int rows = 64);
 int gemm_tc_num_ctas(int row_tiles = 1, int planes = 2);
@@ -80,7 +88,8 @@ PlaneDesc gemm_tc_plan(int n_seg, int seg_cols, int K, bool whole_tiles, long lo
 cudaError_t launch_gemm_tc(const TensorMap *mapX, const TensorMap *const *mapW, int n_seg, int seg_cols, int K,
                            const PlaneDesc &pd, float *P, int ldy, int T, int row0, int32_t *status, cudaStream_t s,
                            int seg0_cols = 0, uint32_t spin_limit = 0, int withhold = 0, int x_row_hi = 0, int x_row_lo = 64,
-                           int row_tiles = 1, int planes = 2, bool serialize = false, int out_t = 0, long long ldt = 0);
+                           int row_tiles = 1, int planes = 2, bool serialize = false, int out_t = 0, long long ldt = 0,
+                           bool packed = false);
 // serialize: launch without programmatic dependent launch.  The kernel requests its streamed ("weight") operand BEFORE it
 // waits for the preceding kernel, which is right for constant weights; a launch whose streamed operand was written by
 // the preceding kernel (the gradient projections of the heads' training) must be fully serialised behind it.

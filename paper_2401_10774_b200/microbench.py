@@ -42,6 +42,7 @@ def main():
     ap.add_argument("--planes", type=int, default=2, choices=(1, 2))
     ap.add_argument("--attention-kernel", type=int, default=0, choices=(0, 1, 2), help="0 automatic, 1 mma.sync, 2 tcgen05")
     ap.add_argument("--no-graphs", action="store_true", help="launch every step kernel by kernel")
+    ap.add_argument("--pack-weights", type=int, default=-1, choices=(-1, 0, 1), help="weights re-laid tile by tile (1) or streamed as given (0); -1: the library's default")
     ap.add_argument("--device-weights", action="store_true",
                     help="draw the weights on the device (N(0, 0.02^2), not the seeded host recipe): seconds instead of a "
                          "minute of set-up, for timing runs whose numbers do not depend on the values")
@@ -87,6 +88,8 @@ def main():
         ctx.set_option(B.OPT_ATTENTION_KERNEL, args.attention_kernel)
     if args.no_graphs:
         ctx.set_option(B.OPT_STEP_GRAPHS, 0)
+    if args.pack_weights >= 0:
+        ctx.set_option(B.OPT_PACK_WEIGHTS, args.pack_weights)
     ctx.load_weights(dw)
     # a cache of the requested length without paying for a long prefill: prefill 64 tokens, then tell the
     # library the rest is there (the K/V values beyond are zeros, which is fine for timing)

@@ -374,6 +374,42 @@ def test_step_graph_replay_matches_plain_launches(oracle, mode):
     assert np.array_equal(kc1, kc0) and np.array_equal(h1, h0)
 
 
+@pytest.mark.parametrize("shape", ["small", "gqa_ragged_ffn", "7b_2layers"])
+def test_packed_weights_give_the_same_bits_as_row_major_weights(shape):
+    """By default a bf16 context streams its own tile-by-tile copy of the backbone matrices (MEDUSA_OPT_PACK_WEIGHTS);
+    the arithmetic and its order are those of the row-major path, so prefill and decode steps must agree bit for bit.
+    The shapes cover matrices whose rows / columns do not fill the last 128 x 64 tile (zero-padded in the packed copy)."""
+    torch, B, U = _gpu()
+    if shape == "small":
+        cfg = I.model_shape("tiny", d=512, n_heads=4, head_dim=128, ffn=1408, vocab=2048, n_medusa=4, n_layers=2)
+    elif shape == "gqa_ragged_ffn":  # ffn 1000: 7.8 tiles of 128 rows and 15.6 k blocks of 64; vocabulary 2000: 15.6 tiles
+        cfg = I.model_shape("tiny", d=512, n_heads=4, n_kv_heads=2, head_dim=128, ffn=1000, vocab=2000, n_medusa=4, n_layers=2)
+    else:
+        cfg = I.model_shape("7b", n_layers=2)
+    w = U.dev_weights(I.make_weights(cfg, seed=21, dtype="bf16", head_init="lm_copy"))
+    prompt = torch.from_numpy(I.make_prompt(150, cfg["vocab"], 22)).cuda()
+    params = B.AcceptParams(mode=B.TYPICAL, temperature=0.7, eps=0.09, delta=0.3)
+    V, d = cfg["vocab"], cfg["d"]
+    runs = []
+    for pack in (1, 0):
+        ctx = U.make_ctx(cfg, "bf16", 512, I.TREE_SPECS["sparse64_d4"])
+        ctx.set_option(B.OPT_PACK_WEIGHTS, pack)
+        ctx.load_weights(w)
+        ctx.prefill(prompt)
+        snaps = []
+        for s in range(5):
+            ctx.decode_step(params)
+            snaps.append((ctx.read_workspace(B.WS_LOGITS, (64, V), np.float32).copy(),
+                          ctx.read_workspace(B.WS_HIDDEN, (64, d), np.float32).copy(), ctx.state()))
+        assert ctx.device_status() == 0
+        runs.append(snaps)
+        ctx.close()
+    for s in range(5):
+        assert np.array_equal(runs[0][s][0].view(np.uint32), runs[1][s][0].view(np.uint32)), "logits differ at step %d" % s
+        assert np.array_equal(runs[0][s][1].view(np.uint32), runs[1][s][1].view(np.uint32)), "hidden differs at step %d" % s
+        assert runs[0][s][2] == runs[1][s][2]
+
+
 def test_bad_acceptance_mode_is_refused_and_leaves_the_step_graphs_on(oracle):
     torch, B, U = _gpu()
     cfg = I.model_shape("tiny")
