@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -85,6 +86,7 @@ struct medusa_ctx {
     int act_planes = 2;
     // MEDUSA_OPT_PACK_WEIGHTS: the weight maps describe the context's own packed copies (packed_on: as loaded)
     bool pack_weights = true, packed_on = false;
+    std::vector<void *> packed_copies;  // the context's packed matrices (also listed in allocs); replaced when weights are loaded anew
     // the lo plane of a split activation (null in the f32 model and when the projections read one plane only)
     void *lo(void *hi, size_t width) const { return m.dtype == MEDUSA_BF16 && act_planes == 2 ? (char *)hi + (size_t)rows * width * 2 : nullptr; }
     // the second plane of q, which the attention kernel reads whatever the projections do
@@ -1062,6 +1064,14 @@ extern "C" int32_t medusa_load_weights(medusa_ctx *c, const medusa_weights *w)
         const int d = m.d, HD = m.n_heads * m.head_dim, HkvD = c->Hkv * m.head_dim, F = m.ffn;
         c->wmaps.resize((size_t)m.n_layers * 7);
         c->packed_on = c->pack_weights;
+        if (!c->packed_copies.empty()) {  // weights loaded anew: the previous packed copies go
+            MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
+            for (void *p : c->packed_copies) {
+                cudaFree(p);
+                c->allocs.erase(std::remove(c->allocs.begin(), c->allocs.end(), p), c->allocs.end());
+            }
+            c->packed_copies.clear();
+        }
         bool ok = true;
         // one matrix: its map over the caller's tensor, or a packed copy of it (kept by the context) and that copy's map
         auto add = [&](TensorMap *tm, const void *W, int N, int K) -> int32_t {
@@ -1071,6 +1081,7 @@ extern "C" int32_t medusa_load_weights(medusa_ctx *c, const medusa_weights *w)
             }
             void *Wp = nullptr;
             TRY(dev_alloc_bytes(c, &Wp, packed_weight_elems(N, K) * 2));
+            c->packed_copies.push_back(Wp);
             launch_pack_weight(W, N, K, Wp, c->stream);
             ok = ok && make_packed_weight_map(tm, Wp, N, K);
             return MEDUSA_OK;

@@ -390,11 +390,7 @@ def test_packed_weights_give_the_same_bits_as_row_major_weights(shape):
     prompt = torch.from_numpy(I.make_prompt(150, cfg["vocab"], 22)).cuda()
     params = B.AcceptParams(mode=B.TYPICAL, temperature=0.7, eps=0.09, delta=0.3)
     V, d = cfg["vocab"], cfg["d"]
-    runs = []
-    for pack in (1, 0):
-        ctx = U.make_ctx(cfg, "bf16", 512, I.TREE_SPECS["sparse64_d4"])
-        ctx.set_option(B.OPT_PACK_WEIGHTS, pack)
-        ctx.load_weights(w)
+    def five_steps(ctx):
         ctx.prefill(prompt)
         snaps = []
         for s in range(5):
@@ -402,12 +398,27 @@ def test_packed_weights_give_the_same_bits_as_row_major_weights(shape):
             snaps.append((ctx.read_workspace(B.WS_LOGITS, (64, V), np.float32).copy(),
                           ctx.read_workspace(B.WS_HIDDEN, (64, d), np.float32).copy(), ctx.state()))
         assert ctx.device_status() == 0
-        runs.append(snaps)
+        return snaps
+
+    runs = []
+    for pack in (1, 0):
+        ctx = U.make_ctx(cfg, "bf16", 512, I.TREE_SPECS["sparse64_d4"])
+        ctx.set_option(B.OPT_PACK_WEIGHTS, pack)
+        ctx.load_weights(w)
+        runs.append(five_steps(ctx))
+        if pack == 0:
+            # the same context loads the weights anew, packed this time (its step graphs and earlier copies are dropped)
+            ctx.set_option(B.OPT_PACK_WEIGHTS, 1)
+            ctx.load_weights(w)
+            runs.append(five_steps(ctx))
+            ctx.load_weights(w)  # and once more: the previous packed copies are released
+            runs.append(five_steps(ctx))
         ctx.close()
-    for s in range(5):
-        assert np.array_equal(runs[0][s][0].view(np.uint32), runs[1][s][0].view(np.uint32)), "logits differ at step %d" % s
-        assert np.array_equal(runs[0][s][1].view(np.uint32), runs[1][s][1].view(np.uint32)), "hidden differs at step %d" % s
-        assert runs[0][s][2] == runs[1][s][2]
+    for other in runs[1:]:
+        for s in range(5):
+            assert np.array_equal(runs[0][s][0].view(np.uint32), other[s][0].view(np.uint32)), "logits differ at step %d" % s
+            assert np.array_equal(runs[0][s][1].view(np.uint32), other[s][1].view(np.uint32)), "hidden differs at step %d" % s
+            assert runs[0][s][2] == other[s][2]
 
 
 def test_bad_acceptance_mode_is_refused_and_leaves_the_step_graphs_on(oracle):
