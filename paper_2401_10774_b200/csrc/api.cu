@@ -32,7 +32,7 @@ struct medusa_ctx {
     float *h_last_all = nullptr, *head_x_all = nullptr, *head_logits_all = nullptr, *gumbel_all = nullptr;
     char *k_cache_all = nullptr, *v_cache_all = nullptr;
     size_t cache_seq_bytes = 0;  // bytes of one sequence's K (or V) cache
-    std::vector<int> L_upper_all;
+    std::vector<int> L_upper_all, L_lower_all;
     int Hkv = 0;  // key/value heads: m.n_kv_heads, or m.n_heads when that is 0 (ordinary multi-head attention)
     cudaStream_t stream = nullptr;
     bool own_stream = false;
@@ -76,6 +76,10 @@ struct medusa_ctx {
     // host-side upper bound of the device-resident cache length (a hint for attention kernels that size their
     // grid on the host; grows by the most a commit can add, exact again after prefill / generate read the length)
     int L_upper = 0;
+    // host-side LOWER bound of the cache length: exact after prefill / generate, and every step adds at least one token.
+    // Which attention kernel a step uses is decided on it, so that the long-cache kernel is only chosen where the cache
+    // really is long (the upper bound drifts away from the length when steps accept less than a full path).
+    int L_lower = 0;
     size_t part_elems = 0;
     float *part = nullptr;  // k-split partial planes of the projection in flight: [planes][64][width]
     // tensor-core path (bf16 model): TMA descriptors of the activation planes and of every weight matrix
@@ -117,6 +121,7 @@ struct medusa_ctx {
     // executable graph, and later steps with that key replay it.  MEDUSA_OPT_STEP_GRAPHS = 0 turns this off.
     struct StepKey {
         int32_t max_commit, has_gumbel, seq;
+        int32_t long_cache;  // whether the step's attention launches are the long-cache kernel's (follows L_lower)
         medusa_accept_params p;
         int32_t *emitted_host, *n_emitted_host;
     };
@@ -233,7 +238,8 @@ void debug_range(medusa_ctx *c, const int32_t *p, int n, int lo, int hi)
 #define DEBUG_RANGE(c, p, n, lo, hi) ((void)0)
 #endif
 
-constexpr int ATTN_TC_MIN_L = 2048;  // measured crossover of the two attention kernels at T = 64, 32 heads
+constexpr int ATTN_TC_MIN_L = 2048;       // measured crossover of the two attention kernels at T = 64, 32 heads, stand-alone
+constexpr int ATTN_TC_STEP_MIN_L = 1536;  // and inside a decode step
 
 enum { PC_GEMM = 0, PC_ATTENTION = 1, PC_HEADS = 2, PC_ELEMWISE = 3, PC_TOPK = 4, PC_POSTERIOR = 5, PC_COMMIT = 6 };
 
@@ -298,17 +304,17 @@ int32_t attention(medusa_ctx *c, const void *q, const void *k_new, const void *v
     const medusa_model_desc &m = c->m;
     if (c->flash_ws) {
         cudaError_t e = cudaSuccess;
-        // Stand-alone, the tcgen05 kernel is the faster one from ATTN_TC_MIN_L cached keys on.  Inside a decode step it
-        // is not: it fills the SM's shared and tensor memory, so the projection that follows cannot stream its first
-        // weight tiles while the attention runs (measured at 7B width up to 3860 keys).
+        // The tcgen05 kernel is the faster one from ATTN_TC_MIN_L cached keys on as a stand-alone operation, and from
+        // ATTN_TC_STEP_MIN_L on inside a decode step (measured at 7B and 13B width: 0.4 % of the step at 1540 keys, 3.6 % at
+        // 2140, 4.6 % at 3900; slower below).  Inside a step the choice follows the host's LOWER bound of the cache length.
         // (the tcgen05 kernel holds one tile of 64 query rows: larger trees always take the mma.sync kernel)
-        if (T <= TREE_ROWS && (c->attn_mode == 2 || (c->attn_mode == 0 && !in_step && L_hint >= ATTN_TC_MIN_L)))
+        if (T <= TREE_ROWS && (c->attn_mode == 2 || (c->attn_mode == 0 && (in_step ? c->L_lower >= ATTN_TC_STEP_MIN_L : L_hint >= ATTN_TC_MIN_L))))
         {
             const int wh = c->withhold == 2 ? 1 : 0;
             if (wh) c->withhold = 0;
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_tc(q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse, c->flash_ws,
                                                                   T, m.n_heads, c->Hkv, m.L_max, L_hint, c->d_state + ST_STATUS, c->stream,
-                                                                  c->spin_limit, wh));
+                                                                  c->spin_limit, wh, q_lo));
         }
         else
             PROF(c, PC_ATTENTION, 1, e = launch_tree_attention_flash(q, k_new, v_new, kc, vc, cache_len, mask, out, out_lo, lse,
@@ -521,6 +527,7 @@ static void point_at(medusa_ctx *c, int b)
     c->k_cache = c->k_cache_all ? c->k_cache_all + (size_t)b * c->cache_seq_bytes : nullptr;
     c->v_cache = c->v_cache_all ? c->v_cache_all + (size_t)b * c->cache_seq_bytes : nullptr;
     if ((size_t)b < c->L_upper_all.size()) c->L_upper = c->L_upper_all[b];
+    if ((size_t)b < c->L_lower_all.size()) c->L_lower = c->L_lower_all[b];
 }
 
 extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc, int32_t device, void *stream)
@@ -553,6 +560,7 @@ extern "C" int32_t medusa_create(medusa_ctx **out, const medusa_model_desc *desc
     c->B = m.max_batch > 1 ? m.max_batch : 1;
     if (c->rows < c->B * TREE_ROWS) c->rows = c->B * TREE_ROWS;  // a batched pass gives every sequence one tile of 64 rows
     c->L_upper_all.assign(c->B, 0);
+    c->L_lower_all.assign(c->B, 0);
     c->stream = (cudaStream_t)stream;
     if (!c->stream) {
         // The legacy default stream cannot be captured into a graph.  A blocking stream orders itself with the
@@ -1111,7 +1119,9 @@ extern "C" int32_t medusa_reset(medusa_ctx *c)
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
     MEDUSA_CUDA(c, cudaMemsetAsync(c->state_all, 0, (size_t)c->B * ST_WORDS * sizeof(int32_t), c->stream));
     c->L_upper_all.assign(c->B, 0);
+    c->L_lower_all.assign(c->B, 0);
     c->L_upper = 0;
+    c->L_lower = 0;
     return MEDUSA_OK;
 }
 
@@ -1136,6 +1146,7 @@ static int32_t prefill_dev(medusa_ctx *c, const int32_t *prompt, int32_t n, int3
         PROF(c, PC_COMMIT,2, launch_commit(m.dtype, a, c->stream));
         MEDUSA_LAUNCH_CHECK(c);
         c->L_upper += T;
+        c->L_lower += T;
     }
     return MEDUSA_OK;
 }
@@ -1149,6 +1160,7 @@ extern "C" int32_t medusa_prefill(medusa_ctx *c, const int32_t *prompt, int32_t 
     MEDUSA_CUDA(c, cudaMemcpyAsync(&L0, c->d_state + ST_CACHE_LEN, sizeof L0, cudaMemcpyDeviceToHost, c->stream));
     MEDUSA_CUDA(c, cudaStreamSynchronize(c->stream));
     c->L_upper = L0;
+    c->L_lower = L0;
     return prefill_dev(c, prompt, n, L0);
 }
 
@@ -1278,6 +1290,7 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
         memset(&key, 0, sizeof key);
         key.max_commit = max_commit;
         key.seq = c->cur;
+        key.long_cache = c->attn_mode == 0 && c->L_lower >= ATTN_TC_STEP_MIN_L ? 1 : 0;
         const bool noisy = gumbel && mode_reads_noise(params);  // the acceptance kernel's own condition
         key.has_gumbel = noisy ? 1 : 0;
         key.p = *params;
@@ -1306,6 +1319,7 @@ extern "C" int32_t medusa_decode_step(medusa_ctx *c, const medusa_accept_params 
         TRY(decode_step_launches(c, params, gumbel, max_commit, emitted_host, n_emitted_host));
     c->L_upper += max_commit;
     if (c->L_upper > m.L_max) c->L_upper = m.L_max;
+    if (c->L_lower < m.L_max) c->L_lower += 1;  // a step that is not refused for a full cache commits at least one token
     return MEDUSA_OK;
 }
 
@@ -1314,6 +1328,7 @@ extern "C" int32_t medusa_select_sequence(medusa_ctx *c, int32_t b)
     if (!c) return MEDUSA_ERR_INVALID_ARG;
     if (b < 0 || b >= c->B) return fail(c, MEDUSA_ERR_INVALID_ARG, "sequence %d: the context holds %d sequence(s)", b, c->B);
     c->L_upper_all[c->cur] = c->L_upper;
+    c->L_lower_all[c->cur] = c->L_lower;
     point_at(c, b);
     c->have_last_key = false;  // the next step belongs to another sequence: its graph is found by the key's sequence index
     return MEDUSA_OK;
@@ -1339,6 +1354,7 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
     MEDUSA_CUDA(c, cudaSetDevice(c->device));
     const int keep = c->cur;
     c->L_upper_all[keep] = c->L_upper;
+    c->L_lower_all[keep] = c->L_lower;
 
     // The launches of a batched step depend on the host through the same values as a single step's (acceptance parameters,
     // commit budget, presence of noise, the host result pointers): the second consecutive batched step with the same key
@@ -1380,6 +1396,7 @@ extern "C" int32_t medusa_decode_step_batch(medusa_ctx *c, const medusa_accept_p
     for (int b = 0; b < B; ++b) {
         const int up = c->L_upper_all[b] + max_commit;
         c->L_upper_all[b] = up > m.L_max ? m.L_max : up;
+        if (c->L_lower_all[b] < m.L_max) c->L_lower_all[b] += 1;
     }
     point_at(c, keep);
     return rc;
@@ -1633,6 +1650,7 @@ extern "C" int32_t medusa_generate(medusa_ctx *c, const int32_t *prompt_host, in
         if (emitted_per_step_host) emitted_per_step_host[steps] = n;
         L += n;
         c->L_upper = L;
+        c->L_lower = L;
         ++steps;
     }
     if (steps_host) *steps_host = steps;

@@ -5,8 +5,13 @@
 // tree's own keys under the ancestor mask).  Per tile two MMAs run entirely out of tensor memory on the A side:
 //     S[128][128]  = Qp[128][128 dims] (TMEM) * K_tile[128 keys][128 dims]^T (shared memory, K-major)
 //     O'[128][128] = P[128][128 keys] (TMEM) * V_tile[128 keys][128 dims]    (shared memory, MN-major)
+// Q is a split activation: both bf16 planes sit in tensor memory and S = Q_hi K^T + Q_lo K^T, so the rounding of q to
+// one plane does not reach the softmax (same accuracy as the mma.sync kernel).  Tensor memory is used to the last
+// column -- two score buffers, the P V accumulator, the two planes of Q -- so P has no region of its own: P of tile
+// i is written over the first 64 columns of the score buffer it was computed from, once both threads of a lane have
+// read their scores, and that buffer takes new scores only after the P V MMA has read P out of it.
 // The 64 query rows are stored twice (TMEM lanes r and 64 + r), and the two copies split every tile's keys: copy 0
-// owns keys 0..63, copy 1 keys 64..127; the other half of a copy's P columns is zero for good.  Each copy keeps
+// owns keys 0..63, copy 1 keys 64..127; the other half of a copy's P columns is written as zero.  Each copy keeps
 // its own running maximum and sum, so the copies never talk during the loop and are merged once at the end like two
 // key ranges.  Two threads share a lane (32 of the copy's 64 keys, 64 of the 128 output columns each) and exchange
 // one partial maximum per tile through shared memory.  The running output stays in registers:
@@ -21,7 +26,7 @@
 // The partial results of the key ranges ([column quad][row][4] floats, so that warps write and read 512 contiguous
 // bytes) are combined by the last CTA of a head to arrive (ticket), in range order; the workspace has the size of
 // the mma.sync kernel's (attention_flash.cu).  In steady state the loop streams K/V at ~6 TB/s; the kernel is the
-// faster of the two from about 2048 cached keys on.
+// faster of the two from about 2048 cached keys on as a stand-alone operation and from about 1536 inside a decode step.
 #include <cuda.h>
 
 #include <unordered_map>
@@ -47,11 +52,13 @@ constexpr int TAIL_BYTES = 4096;         // barriers and exchange buffers (struc
 constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + TAIL_BYTES;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t O_COL = 256, P_COL = 384, Q_COL = 448;  // S0: 0..127, S1: 128..255, O': 256..383, P: 384..447, Q: 448..511
+// S0: 0..127, S1: 128..255, O': 256..383, Q lo plane: 384..447, Q hi plane: 448..511.  P of tile i is written over the
+// first 64 columns of the score buffer S(i & 1) it was computed from, once both threads of a lane have read their scores.
+constexpr uint32_t O_COL = 256, QLO_COL = 384, Q_COL = 448;
 constexpr int MAX_SPLITS = FLASH_MAX_SPLITS;
 
 struct Smem {
-    uint64_t kv_full[STAGES], kv_empty[STAGES], s_full[2], s_empty[2], p_full, p_empty, o_full, o_empty, q_full, done;
+    uint64_t kv_full[STAGES], kv_empty[STAGES], s_full[2], s_empty[2], p_full, o_full, o_empty, q_full, done;
     uint32_t tmem_base;
     volatile int failed;
     int ticket;
@@ -229,7 +236,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 struct Args {
-    const bf16 *q, *k_new, *v_new;   // [T][H][D]
+    const bf16 *q, *q_lo, *k_new, *v_new;   // [T][H][D]; q_lo (nullable): the second bf16 plane of a split q
     const bf16 *k_cache, *v_cache;   // [H][L_max][D]
     const int32_t *cache_len;
     const uint64_t *mask;            // [T]
@@ -275,10 +282,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm->s_full[b], 1);
-            mbar_init(&sm->s_empty[b], 8);   // one arrival per softmax warp
+            mbar_init(&sm->s_empty[b], 1);   // tcgen05.commit of the P V MMA that read this buffer's P
         }
         mbar_init(&sm->p_full, 8);
-        mbar_init(&sm->p_empty, 1);
         mbar_init(&sm->o_full, 1);
         mbar_init(&sm->o_empty, 8);
         mbar_init(&sm->q_full, 8);
@@ -299,13 +305,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
     for (int i = 0; i < 64; ++i)
         o[i] = 0.f;
     // Q row r, dims hf*64..: requested now, stored to tensor memory once that is allocated
-    uint32_t qv[32];
+    uint32_t qv[32], qlv[32];
+    const bool has_qlo = a.q_lo != nullptr;
     if (softmax_warp) {
-        const uint4 *src = reinterpret_cast<const uint4 *>(a.q + (size_t)min(r, a.T - 1) * HD + (size_t)h * D + hf * 64);
+        const size_t qoff = (size_t)min(r, a.T - 1) * HD + (size_t)h * D + hf * 64;
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.q + qoff);
+        const uint4 *src_lo = reinterpret_cast<const uint4 *>((has_qlo ? a.q_lo : a.q) + qoff);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint4 v = r < a.T ? src[j] : make_uint4(0u, 0u, 0u, 0u);
             qv[4 * j] = v.x; qv[4 * j + 1] = v.y; qv[4 * j + 2] = v.z; qv[4 * j + 3] = v.w;
+            const uint4 u = r < a.T && has_qlo ? src_lo[j] : make_uint4(0u, 0u, 0u, 0u);
+            qlv[4 * j] = u.x; qlv[4 * j + 1] = u.y; qlv[4 * j + 2] = u.z; qlv[4 * j + 3] = u.w;
         }
     }
     uint32_t tmem = 0;
@@ -382,7 +393,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
             mbar_wait(&sm->q_full, 0, failed, a.spin_limit);  // Q sits in tensor memory
             for (int i = 0; i < n_tiles; ++i) {
                 mbar_wait(&sm->kv_full[i % STAGES], (i / STAGES) & 1, failed, a.spin_limit);
-                if (i >= 2)
+                if (i >= 2)  // the P V MMA of tile i - 2 has read its P out of this buffer
                     mbar_wait(&sm->s_empty[i & 1], ((i >> 1) - 1) & 1, failed, a.spin_limit);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t dk = desc_kmajor(smem_u32(ring + (i % STAGES) * STAGE_BYTES));
@@ -391,6 +402,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
                 for (int ks = 0; ks < 8; ++ks) {  // 16 dims per step: 8 packed columns of Q, 32 bytes inside a K row
                     const uint64_t ko = (uint64_t)(((ks >> 2) * KSUB_BYTES + (ks & 3) * 32) >> 4);
                     umma_ts(td, tmem + Q_COL + (uint32_t)(ks * 8), dk + ko, IDESC_S, ks ? 1u : 0u, leader);
+                }
+                if (has_qlo) {  // S += Q_lo K^T: q's rounding to one bf16 plane does not reach the softmax
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t ko = (uint64_t)(((ks >> 2) * KSUB_BYTES + (ks & 3) * 32) >> 4);
+                        umma_ts(td, tmem + QLO_COL + (uint32_t)(ks * 8), dk + ko, IDESC_S, 1u, leader);
+                    }
                 }
                 umma_commit(&sm->s_full[i & 1], leader);
             }
@@ -403,9 +421,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
                 const uint64_t dv = desc_mnmajor(smem_u32(ring + (i % STAGES) * STAGE_BYTES) + K_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < BKEY / 16; ++kk)  // 16 keys per step: 8 packed columns of P, 16 V rows of 128 bytes
-                    umma_ts(tmem + O_COL, tmem + P_COL + (uint32_t)(kk * 8), dv + (uint64_t)((kk * 2048) >> 4), IDESC_O, kk ? 1u : 0u,
-                            leader);
-                umma_commit(&sm->p_empty, leader);
+                    umma_ts(tmem + O_COL, tmem + (uint32_t)((i & 1) * BKEY + kk * 8), dv + (uint64_t)((kk * 2048) >> 4), IDESC_O,
+                            kk ? 1u : 0u, leader);
+                umma_commit(&sm->s_empty[i & 1], leader);  // P has been read: the buffer may take the scores of tile i + 2
                 umma_commit(&sm->o_full, leader);
                 umma_commit(&sm->kv_empty[i % STAGES], leader);  // the scores of this stage were read before its P existed
             }
@@ -426,14 +444,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
         const uint64_t mask_r = r < a.T ? a.mask[r] : 0ull;
         const float sc = rsqrtf((float)D) * LOG2E;
         {
-            // Q: 32 packed columns of this thread's lane; the other copy's P columns are zero for good
+            // Q: 32 packed columns of this thread's lane in each plane
             tmem_st16(tmem + lane_addr + Q_COL + (uint32_t)(hf * 32), qv);
             tmem_st16(tmem + lane_addr + Q_COL + (uint32_t)(hf * 32 + 16), qv + 16);
-            uint32_t z[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                z[j] = 0u;
-            tmem_st16(tmem + lane_addr + P_COL + (uint32_t)((1 - copy) * 32 + hf * 16), z);
+            tmem_st16(tmem + lane_addr + QLO_COL + (uint32_t)(hf * 32), qlv);
+            tmem_st16(tmem + lane_addr + QLO_COL + (uint32_t)(hf * 32 + 16), qlv + 16);
             tmem_st_wait();
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -448,10 +463,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
                 mbar_wait(&sm->s_full[i & 1], (i >> 1) & 1, failed, a.spin_limit);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 tmem_ld32(tmem + lane_addr + (uint32_t)((i & 1) * BKEY + copy * 64 + hf * 32), s);
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0)
-                    mbar_arrive(&sm->s_empty[i & 1]);
                 const int ct = tile0 + i;
                 const bool tree_tile = ct >= tile1;
                 const int kj0 = copy * 64 + hf * 32;  // first key of this thread inside the tile
@@ -485,10 +496,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
                     pk[j] = pack_bf16(p0, p1);
                 }
                 l = l * c + (ps0 + ps1);
-                if (i >= 1)
-                    mbar_wait(&sm->p_empty, (i - 1) & 1, failed, a.spin_limit);  // the previous tile's P V has read P
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                tmem_st16(tmem + lane_addr + P_COL + (uint32_t)(copy * 32 + hf * 16), pk);
+                // P goes over the first 64 columns of the score buffer it came from: both threads of this lane have read
+                // their scores (they met on the copy's barrier above), and the buffer is not written again before the
+                // P V MMA of this tile has read P.  The half that belongs to the other copy's keys is zero.
+                {
+                    uint32_t z[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        z[j] = 0u;
+                    tmem_st16(tmem + lane_addr + (uint32_t)((i & 1) * BKEY + copy * 32 + hf * 16), pk);
+                    tmem_st16(tmem + lane_addr + (uint32_t)((i & 1) * BKEY + (1 - copy) * 32 + hf * 16), z);
+                }
                 tmem_st_wait();
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
@@ -666,7 +684,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                      const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                      void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                     int L_hint, int32_t *status, cudaStream_t s, uint32_t spin_limit, int withhold)
+                                     int L_hint, int32_t *status, cudaStream_t s, uint32_t spin_limit, int withhold,
+                                     const void *q_lo)
 {
     // TMA descriptors of the two caches ([Hkv * L_max rows][128 dims] bf16, boxes of 64 dims x 128 rows), encoded once
     // per distinct cache
@@ -709,7 +728,7 @@ cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const voi
         splits = (nt + tps - 1) / tps;
     }
     Args a;
-    a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
+    a.q = (const bf16 *)q; a.q_lo = (const bf16 *)q_lo; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
     a.k_cache = (const bf16 *)k_cache; a.v_cache = (const bf16 *)v_cache;
     a.cache_len = cache_len; a.mask = mask; a.out = (bf16 *)out; a.out_lo = (bf16 *)out_lo; a.lse = lse;
     a.ws_o = (float *)workspace;

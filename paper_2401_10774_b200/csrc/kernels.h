@@ -71,7 +71,8 @@ cudaError_t launch_tree_attention_flash(const void *q, const void *k_new, const 
 cudaError_t launch_tree_attention_tc(const void *q, const void *k_new, const void *v_new, const void *k_cache,
                                      const void *v_cache, const int32_t *cache_len, const uint64_t *mask, void *out,
                                      void *out_lo, float *lse, void *workspace, int T, int H, int Hkv, int L_max,
-                                     int L_hint, int32_t *status, cudaStream_t s, uint32_t spin_limit = 0, int withhold = 0);
+                                     int L_hint, int32_t *status, cudaStream_t s, uint32_t spin_limit = 0, int withhold = 0,
+                                     const void *q_lo = nullptr);
 
 // ---- heads.cu ----
 // x_k = h + SiLU(W1_k h) -> float [K][d];  h: float if h_is_f32 else the model dtype
