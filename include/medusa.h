@@ -133,7 +133,10 @@ enum {
 /* Context options for medusa_set_option. */
 enum {
     MEDUSA_OPT_STEP_GRAPHS = 0,      /* 1 (default): medusa_decode_step may capture and replay whole-step CUDA graphs; 0: never */
-    MEDUSA_OPT_ATTENTION_KERNEL = 1, /* bf16 / head_dim 128 tree attention: 0 automatic (default), 1 mma.sync, 2 tcgen05 */
+    MEDUSA_OPT_ATTENTION_KERNEL = 1, /* bf16 / head_dim 128 tree attention: 1 mma.sync, 2 tcgen05, 0 (default) automatic: the
+                                      * tcgen05 kernel for trees of up to 64 nodes from 2048 cached keys on in
+                                      * medusa_tree_attention (by the length hint) and from 1536 on inside a pass or step (by
+                                      * the host's lower bound of the cache length: exact after prefill, +1 per step) */
     MEDUSA_OPT_ATTENTION_LENGTH_HINT = 2, /* host-side upper bound of *cache_len for medusa_tree_attention (kernel choice and
                                            * grid size follow it; a longer cache is still processed completely); < 0: L_max */
     MEDUSA_OPT_LAYER_TAP = 3,        /* layer whose input / attention output / output the next passes copy to the TAP
