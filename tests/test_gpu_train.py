@@ -20,6 +20,7 @@ CASES = [
     ("small_2heads_77", 256, 1024, 2, 77, 0.05),
     ("small_2heads_2chunks_1324", 512, 2048, 2, 1324, 0.05),
     ("7b_width_1head_300", 4096, 32000, 1, 300, 0.02),
+    ("13b_width_2heads_2chunks_1100", 5120, 32000, 2, 1100, 0.02),
 ]
 
 
